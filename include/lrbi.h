@@ -1,0 +1,152 @@
+/*
+ * lrbi -- inference with a layer pruned by a tiled low-rank binary index (B200, sm_100a).
+ *
+ * Plain C ABI.  The pruning index of a layer W [rows x cols] (rows = output features,
+ * cols = input features) is not stored; it is rebuilt from two small binary factors per
+ * tile.  The index matrix is cut into equal tiles of tile_rows x tile_cols (Section 3.1
+ * of the paper: each block is factorised, hence decoded, independently, all with the same
+ * rank k).  For tile (tr, tc) with factors Ip (tile_rows x k) and Iz (k x tile_cols) the
+ * decoded index is the Boolean matrix product of Eq. 3,
+ *
+ *        Ia[i][j] = OR_{l=1..k} ( Ip[i][l] AND Iz[l][j] ),
+ *
+ * where a 1 keeps the weight and a 0 prunes it to zero (Section 2, Eq. 1-2).  Ia is the
+ * masking layer of the layer (Sections 2 and 2.2), so the layer computes
+ * Y = X * (W .* Ia)^T.
+ *
+ * Packed factor format (KW = ceil(k / 32) 32-bit words per row of Ip / per column of Iz,
+ * GR = ceil(rows / tile_rows), GC = ceil(cols / tile_cols), tile index t = tr * GC + tc):
+ *
+ *   ip[(t * tile_rows + i) * KW + w]   bit (l % 32) of word w = l / 32   is  Ip_t[i][l]
+ *   iz[(t * tile_cols + j) * KW + w]   bit (l % 32) of word w = l / 32   is  Iz_t[l][j]
+ *
+ * Edge tiles still hold tile_rows row words and tile_cols column words; those that fall
+ * outside the matrix are ignored.  Bits at positions >= k of the last word are ignored.
+ *
+ * Unless an argument says "host", every pointer is a DEVICE pointer owned by the caller,
+ * valid on the current device, 16-byte aligned.  Calls are asynchronous and ordered on
+ * `stream` (a cudaStream_t passed as void*, NULL = the legacy default stream).  Inputs are
+ * only read.  Nothing outside the stated output extent is written.  Argument errors are
+ * detected on the host before anything is launched and reported by the return code; no
+ * call aborts, throws or traps.  There is no CPU fallback: without a usable sm_100 device
+ * a compute call returns LRBI_ERR_CUDA.
+ */
+#ifndef LRBI_H_
+#define LRBI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LRBI_API __attribute__((visibility("default")))
+#else
+#define LRBI_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LRBI_OK = 0,
+    LRBI_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer          */
+    LRBI_ERR_UNSUPPORTED = 2, /* a shape, dtype or kernel choice this build does not cover     */
+    LRBI_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed (see lrbi_last_cuda_error)  */
+    LRBI_ERR_TIMEOUT = 4      /* a bounded device-side wait gave up (see lrbi_device_status)   */
+} lrbi_status;
+
+/* Geometry of one pruned layer (Section 3.1: equal tiles, one rank). */
+typedef struct {
+    int32_t rows;      /* output features: rows of W and of the index          */
+    int32_t cols;      /* input features: columns of W and of the index        */
+    int32_t tile_rows; /* tm >= 1                                               */
+    int32_t tile_cols; /* tn >= 1                                               */
+    int32_t rank;      /* k >= 1, the same for every tile                       */
+} lrbi_layout;
+
+/* Output element type of lrbi_masked_gemm. */
+enum { LRBI_Y_BF16 = 0, LRBI_Y_F32 = 1 };
+
+/* Kernel choice for lrbi_masked_gemm / lrbi_decode_mask (LRBI_ALGO_AUTO picks by shape). */
+enum {
+    LRBI_ALGO_AUTO = 0,
+    LRBI_ALGO_GENERIC = 1,   /* any shape; one thread per output, slow                         */
+    LRBI_ALGO_GEMV = 2,      /* small batch, bandwidth-bound, CUDA-core FMA                    */
+    LRBI_ALGO_TENSOR = 3,    /* tcgen05 MMA with TMEM accumulators                             */
+    LRBI_ALGO_DECODE_BALLOT = 4, /* decode: one __ballot_sync per 32-bit mask word             */
+    LRBI_ALGO_DECODE_PLANES = 5  /* decode: ballot-transposed Iz bit-planes, OR per 32 columns */
+};
+
+/* Element counts of the packed arrays for a layout (0 if the layout is invalid). */
+LRBI_API size_t lrbi_packed_ip_words(const lrbi_layout *layout); /* GR*GC*tile_rows*KW */
+LRBI_API size_t lrbi_packed_iz_words(const lrbi_layout *layout); /* GR*GC*tile_cols*KW */
+LRBI_API size_t lrbi_mask_words(const lrbi_layout *layout);      /* rows*ceil(cols/32) */
+
+/*
+ * Decode the whole index (Eq. 3 per tile, Section 3.1) into a bit-packed mask.
+ *   ip, iz    device, packed factors as above (read only)
+ *   mask_out  device, rows x ceil(cols/32) uint32, row-major; bit (c % 32) of word c / 32
+ *             of row r is Ia[r][c]; bits beyond `cols` in the last word of a row are 0.
+ *   algo      LRBI_ALGO_AUTO, LRBI_ALGO_DECODE_BALLOT or LRBI_ALGO_DECODE_PLANES
+ *             (PLANES needs tile_cols % 32 == 0, else LRBI_ERR_UNSUPPORTED)
+ * Every word of mask_out is written; nothing else is.
+ */
+LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t *ip, const uint32_t *iz,
+                             uint32_t *mask_out, int32_t algo, void *stream);
+
+/*
+ * Fused decode + prune + dense product (Eq. 3; masking layer of Sections 2 and 2.2):
+ *       Y[b][o] = sum_i  Ia[o][i] ? X[b][i] * W[o][i] : 0      (fp32 accumulation)
+ * The decoded index never reaches device memory.  A pruned weight is selected away, not
+ * multiplied by zero, so a NaN/Inf stored in a pruned position does not reach Y.
+ *   W      device, bf16 bit patterns, [rows][cols] row-major
+ *   X      device, bf16 bit patterns, [batch][cols] row-major
+ *   Y      device, [batch][rows] row-major, bf16 (round to nearest even) or fp32 per y_dtype
+ *   algo   LRBI_ALGO_AUTO, _GENERIC, _GEMV (batch <= 8) or _TENSOR; a kernel that does not
+ *          cover the shape returns LRBI_ERR_UNSUPPORTED and launches nothing.
+ * The tensor-core path may split the reduction over several thread blocks; it then keeps
+ * fp32 partial sums in a library-owned device buffer that grows (cudaMalloc) on the first
+ * call that needs more, so such a first call must not be made during stream capture.
+ * Calls that use that buffer concurrently on different streams are not supported.
+ */
+LRBI_API lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const uint32_t *ip,
+                             const uint32_t *iz, const uint16_t *X, int32_t batch, void *Y,
+                             int32_t y_dtype, int32_t algo, void *stream);
+
+/*
+ * Same computation for callers whose activations live in host memory (the index and the
+ * weights are uploaded once, activations and results cross the bus on every call).
+ *   lrbi_layer_create   copies W, ip, iz (HOST pointers) to the current device and reserves
+ *                       staging for up to max_batch rows.  *out owns device memory.
+ *   lrbi_layer_forward_host   X_host [batch][cols] bf16 and Y_host [batch][rows] are HOST
+ *                       pointers (pinned memory makes the copies asynchronous and overlapped
+ *                       with the kernels, chunk by chunk); returns after Y_host is complete.
+ *   lrbi_layer_destroy  frees everything the handle owns.
+ */
+typedef struct lrbi_layer lrbi_layer;
+LRBI_API lrbi_status lrbi_layer_create(const lrbi_layout *layout, const uint16_t *W_host,
+                              const uint32_t *ip_host, const uint32_t *iz_host,
+                              int32_t max_batch, lrbi_layer **out);
+LRBI_API lrbi_status lrbi_layer_forward_host(lrbi_layer *layer, const uint16_t *X_host, int32_t batch,
+                                    void *Y_host, int32_t y_dtype, int32_t algo);
+LRBI_API lrbi_status lrbi_layer_destroy(lrbi_layer *layer);
+
+/* Which kernel LRBI_ALGO_AUTO would run for this layout and batch (an LRBI_ALGO_* value). */
+LRBI_API int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batch);
+
+/* Kernels launched by this library since it was loaded (all entry points, this process). */
+LRBI_API uint64_t lrbi_launch_count(void);
+
+/*
+ * Device-side status word of the current device: 0, or a code left by a kernel whose bounded
+ * wait (pipeline barrier) ran out.  Synchronises the device.  `clear` != 0 resets it.
+ */
+LRBI_API int32_t lrbi_device_status(int32_t clear);
+
+LRBI_API const char *lrbi_status_string(lrbi_status s);
+LRBI_API int32_t lrbi_last_cuda_error(void); /* cudaError_t / CUresult of the last failed call, else 0 */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LRBI_H_ */

@@ -1,0 +1,205 @@
+"""Python binding of the lrbi C ABI: argument marshalling only.
+
+Every step of the path (decode, pruning, product) runs in the CUDA library; this module turns
+torch CUDA tensors into device pointers and checks return codes.  torch is used for device
+memory and streams.  If the library is not built, importing a compute function's first call
+raises: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+from .synth import Layer
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblrbi.so")
+
+ALGO_AUTO, ALGO_GENERIC, ALGO_GEMV, ALGO_TENSOR, ALGO_DECODE_BALLOT, ALGO_DECODE_PLANES = range(6)
+ALGO_NAMES = {0: "auto", 1: "generic", 2: "gemv", 3: "tensor", 4: "decode_ballot", 5: "decode_planes"}
+Y_BF16, Y_F32 = 0, 1
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = range(5)
+
+
+class LrbiError(RuntimeError):
+    def __init__(self, code, what):
+        self.code = code
+        super().__init__("%s: %s (status %d, cuda error %d)" % (what, status_string(code), code, lib().lrbi_last_cuda_error()))
+
+
+class Layout(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int32), ("cols", ctypes.c_int32), ("tile_rows", ctypes.c_int32),
+                ("tile_cols", ctypes.c_int32), ("rank", ctypes.c_int32)]
+
+    @classmethod
+    def of(cls, layer):
+        if isinstance(layer, cls):
+            return layer
+        if isinstance(layer, Layer):
+            return cls(layer.rows, layer.cols, layer.tile_rows, layer.tile_cols, layer.rank)
+        return cls(*layer)
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("lrbi CUDA library missing: %s (run paper_1905_05686_b200/build.py); "
+                               "there is no CPU fallback" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, lp = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Layout)
+        for name in ("lrbi_packed_ip_words", "lrbi_packed_iz_words", "lrbi_mask_words"):
+            getattr(L, name).argtypes = [lp]
+            getattr(L, name).restype = ctypes.c_size_t
+        L.lrbi_decode_mask.argtypes = [lp, vp, vp, vp, i32, vp]
+        L.lrbi_decode_mask.restype = i32
+        L.lrbi_masked_gemm.argtypes = [lp, vp, vp, vp, vp, i32, vp, i32, i32, vp]
+        L.lrbi_masked_gemm.restype = i32
+        L.lrbi_layer_create.argtypes = [lp, vp, vp, vp, i32, ctypes.POINTER(vp)]
+        L.lrbi_layer_create.restype = i32
+        L.lrbi_layer_forward_host.argtypes = [vp, vp, i32, vp, i32, i32]
+        L.lrbi_layer_forward_host.restype = i32
+        L.lrbi_layer_destroy.argtypes = [vp]
+        L.lrbi_layer_destroy.restype = i32
+        L.lrbi_masked_gemm_choice.argtypes = [lp, i32]
+        L.lrbi_masked_gemm_choice.restype = i32
+        L.lrbi_launch_count.argtypes = []
+        L.lrbi_launch_count.restype = ctypes.c_uint64
+        L.lrbi_device_status.argtypes = [i32]
+        L.lrbi_device_status.restype = i32
+        L.lrbi_status_string.argtypes = [i32]
+        L.lrbi_status_string.restype = ctypes.c_char_p
+        L.lrbi_last_cuda_error.argtypes = []
+        L.lrbi_last_cuda_error.restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().lrbi_status_string(code).decode()
+
+
+def launch_count() -> int:
+    return int(lib().lrbi_launch_count())
+
+
+def device_status(clear: bool = False) -> int:
+    return int(lib().lrbi_device_status(1 if clear else 0))
+
+
+def masked_gemm_choice(layer, batch: int) -> int:
+    lay = Layout.of(layer)
+    return int(lib().lrbi_masked_gemm_choice(ctypes.byref(lay), batch))
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, what):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (what, dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def to_device_words(a: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint32 numpy words -> int32 CUDA tensor holding the same bits."""
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint32).view(np.int32)).to(device)
+
+
+def to_device_bf16(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bf16 bit patterns -> bfloat16 CUDA tensor holding the same bits."""
+    return torch.from_numpy(np.ascontiguousarray(bits, dtype=np.uint16).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def lrbi_decode_mask(layer, ip: torch.Tensor, iz: torch.Tensor, mask_out: torch.Tensor | None = None,
+                     algo: int = ALGO_AUTO, stream=None) -> torch.Tensor:
+    """Bit-packed decoded index [rows, ceil(cols/32)] (int32 tensor holding uint32 words)."""
+    lay = Layout.of(layer)
+    L = lib()
+    if ip.numel() != L.lrbi_packed_ip_words(ctypes.byref(lay)) or iz.numel() != L.lrbi_packed_iz_words(ctypes.byref(lay)):
+        raise ValueError("packed factor sizes do not match the layout")
+    if mask_out is None:
+        mask_out = torch.empty((lay.rows, (lay.cols + 31) // 32), dtype=torch.int32, device=ip.device)
+    elif mask_out.numel() != L.lrbi_mask_words(ctypes.byref(lay)):
+        raise ValueError("mask_out has the wrong size")
+    rc = L.lrbi_decode_mask(ctypes.byref(lay), _dev(ip, torch.int32, "ip"), _dev(iz, torch.int32, "iz"),
+                            _dev(mask_out, torch.int32, "mask_out"), algo, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_decode_mask")
+    return mask_out
+
+
+def lrbi_masked_gemm(layer, W: torch.Tensor, ip: torch.Tensor, iz: torch.Tensor, X: torch.Tensor,
+                     Y: torch.Tensor | None = None, y_dtype=torch.bfloat16, algo: int = ALGO_AUTO,
+                     stream=None) -> torch.Tensor:
+    """Y = X (W .* Ia)^T with the index decoded on the fly; W [rows, cols], X [batch, cols] bf16."""
+    lay = Layout.of(layer)
+    L = lib()
+    if tuple(W.shape) != (lay.rows, lay.cols) or X.dim() != 2 or X.shape[1] != lay.cols:
+        raise ValueError("W / X shapes do not match the layout")
+    if ip.numel() != L.lrbi_packed_ip_words(ctypes.byref(lay)) or iz.numel() != L.lrbi_packed_iz_words(ctypes.byref(lay)):
+        raise ValueError("packed factor sizes do not match the layout")
+    batch = X.shape[0]
+    if Y is None:
+        Y = torch.empty((batch, lay.rows), dtype=y_dtype, device=X.device)
+    if tuple(Y.shape) != (batch, lay.rows) or Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be [batch, rows] bf16 or fp32")
+    code = Y_BF16 if Y.dtype == torch.bfloat16 else Y_F32
+    rc = L.lrbi_masked_gemm(ctypes.byref(lay), _dev(W, torch.bfloat16, "W"), _dev(ip, torch.int32, "ip"),
+                            _dev(iz, torch.int32, "iz"), _dev(X, torch.bfloat16, "X"), batch,
+                            _dev(Y, Y.dtype, "Y"), code, algo, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_masked_gemm")
+    return Y
+
+
+class HostLayer:
+    """lrbi_layer_* handle: weights and index resident on the device, activations from host memory."""
+
+    def __init__(self, layer, W_bits: np.ndarray, ip_words: np.ndarray, iz_words: np.ndarray, max_batch: int):
+        self.layout = Layout.of(layer)
+        W_bits = np.ascontiguousarray(W_bits, dtype=np.uint16)
+        ip_words = np.ascontiguousarray(ip_words, dtype=np.uint32)
+        iz_words = np.ascontiguousarray(iz_words, dtype=np.uint32)
+        h = ctypes.c_void_p()
+        rc = lib().lrbi_layer_create(ctypes.byref(self.layout), W_bits.ctypes.data, ip_words.ctypes.data,
+                                     iz_words.ctypes.data, max_batch, ctypes.byref(h))
+        if rc != OK:
+            raise LrbiError(rc, "lrbi_layer_create")
+        self._h = h
+
+    def forward_host(self, X_host: torch.Tensor, Y_host: torch.Tensor, algo: int = ALGO_AUTO):
+        """X_host [batch, cols] bf16 and Y_host [batch, rows] bf16/fp32 are CPU tensors (pinned for overlap)."""
+        if X_host.is_cuda or Y_host.is_cuda or not X_host.is_contiguous() or not Y_host.is_contiguous():
+            raise TypeError("forward_host takes contiguous CPU tensors")
+        if X_host.dtype != torch.bfloat16 or X_host.shape[1] != self.layout.cols:
+            raise ValueError("X_host must be [batch, cols] bf16")
+        batch = X_host.shape[0]
+        if tuple(Y_host.shape) != (batch, self.layout.rows):
+            raise ValueError("Y_host must be [batch, rows]")
+        code = Y_BF16 if Y_host.dtype == torch.bfloat16 else Y_F32
+        rc = lib().lrbi_layer_forward_host(self._h, ctypes.c_void_p(X_host.data_ptr()), batch,
+                                           ctypes.c_void_p(Y_host.data_ptr()), code, algo)
+        if rc != OK:
+            raise LrbiError(rc, "lrbi_layer_forward_host")
+        return Y_host
+
+    def close(self):
+        if self._h:
+            lib().lrbi_layer_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

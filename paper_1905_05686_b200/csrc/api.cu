@@ -1,0 +1,259 @@
+// C ABI of the lrbi library: argument checks, kernel choice, host-buffer layer handle.
+#include <atomic>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "lrbi_common.cuh"
+
+namespace lrbi {
+
+__device__ int g_device_status = 0;
+
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_last_cuda_error{0};
+static std::mutex g_mutex;
+static int *g_status_ptr[64] = {nullptr};
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+void note_cuda_error(int code) { g_last_cuda_error.store(code, std::memory_order_relaxed); }
+
+int *device_status_ptr()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_status_ptr[dev]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_device_status);
+        if (e != cudaSuccess) { note_cuda_error((int)e); return nullptr; }
+        g_status_ptr[dev] = static_cast<int *>(p);
+    }
+    return g_status_ptr[dev];
+}
+
+static bool layout_ok(const lrbi_layout *l)
+{
+    if (!l) return false;
+    if (l->rows < 1 || l->cols < 1 || l->tile_rows < 1 || l->tile_cols < 1 || l->rank < 1) return false;
+    return true;
+}
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int choose_gemm(const Geo &g, int batch)
+{
+    if (batch <= 8 && gemv_supported(g, batch)) return LRBI_ALGO_GEMV;
+    if (gemm_tc_supported(g, batch)) return LRBI_ALGO_TENSOR;
+    return LRBI_ALGO_GENERIC;
+}
+
+}  // namespace lrbi
+
+using namespace lrbi;
+
+extern "C" {
+
+size_t lrbi_packed_ip_words(const lrbi_layout *l)
+{
+    if (!layout_ok(l)) return 0;
+    Geo g = make_geo(*l);
+    return (size_t)g.gr * g.gc * g.tm * g.kw;
+}
+size_t lrbi_packed_iz_words(const lrbi_layout *l)
+{
+    if (!layout_ok(l)) return 0;
+    Geo g = make_geo(*l);
+    return (size_t)g.gr * g.gc * g.tn * g.kw;
+}
+size_t lrbi_mask_words(const lrbi_layout *l)
+{
+    if (!layout_ok(l)) return 0;
+    Geo g = make_geo(*l);
+    return (size_t)g.rows * g.pitch;
+}
+
+lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t *ip, const uint32_t *iz,
+                             uint32_t *mask_out, int32_t algo, void *stream)
+{
+    if (!layout_ok(layout) || !ip || !iz || !mask_out) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(ip) || !aligned16(iz) || !aligned16(mask_out)) return LRBI_ERR_INVALID_ARG;
+    const Geo g = make_geo(*layout);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (algo) {
+    case LRBI_ALGO_AUTO:
+        return decode_planes_supported(g) ? launch_decode_planes(g, ip, iz, mask_out, s)
+                                          : launch_decode_ballot(g, ip, iz, mask_out, s);
+    case LRBI_ALGO_DECODE_BALLOT: return launch_decode_ballot(g, ip, iz, mask_out, s);
+    case LRBI_ALGO_DECODE_PLANES: return launch_decode_planes(g, ip, iz, mask_out, s);
+    default: return LRBI_ERR_INVALID_ARG;
+    }
+}
+
+int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batch)
+{
+    if (!layout_ok(layout) || batch < 1) return -1;
+    return choose_gemm(make_geo(*layout), batch);
+}
+
+lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const uint32_t *ip,
+                             const uint32_t *iz, const uint16_t *X, int32_t batch, void *Y,
+                             int32_t y_dtype, int32_t algo, void *stream)
+{
+    if (!layout_ok(layout) || !W || !ip || !iz || !X || !Y || batch < 1) return LRBI_ERR_INVALID_ARG;
+    if (y_dtype != LRBI_Y_BF16 && y_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(ip) || !aligned16(iz) || !aligned16(X) || !aligned16(Y)) return LRBI_ERR_INVALID_ARG;
+    const Geo g = make_geo(*layout);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (algo == LRBI_ALGO_AUTO) algo = choose_gemm(g, batch);
+    switch (algo) {
+    case LRBI_ALGO_GENERIC: return launch_gemm_generic(g, W, ip, iz, X, batch, Y, y_dtype, s);
+    case LRBI_ALGO_GEMV: return launch_gemv(g, W, ip, iz, X, batch, Y, y_dtype, s);
+    case LRBI_ALGO_TENSOR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s);
+    default: return LRBI_ERR_INVALID_ARG;
+    }
+}
+
+uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int32_t lrbi_device_status(int32_t clear)
+{
+    int *p = device_status_ptr();
+    if (!p) return -1;
+    int v = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&v, p, sizeof v, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { note_cuda_error((int)e); return -1; }
+    if (clear && v != 0) {
+        const int zero = 0;
+        cudaMemcpy(p, &zero, sizeof zero, cudaMemcpyHostToDevice);
+    }
+    return v;
+}
+
+const char *lrbi_status_string(lrbi_status s)
+{
+    switch (s) {
+    case LRBI_OK: return "ok";
+    case LRBI_ERR_INVALID_ARG: return "invalid argument";
+    case LRBI_ERR_UNSUPPORTED: return "unsupported shape or kernel choice";
+    case LRBI_ERR_CUDA: return "CUDA call failed";
+    case LRBI_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+    }
+}
+
+int32_t lrbi_last_cuda_error(void) { return g_last_cuda_error.load(std::memory_order_relaxed); }
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer layer handle
+// ---------------------------------------------------------------------------------------------
+struct lrbi_layer {
+    lrbi_layout layout;
+    Geo g;
+    int max_batch;
+    uint16_t *W = nullptr;
+    uint32_t *ip = nullptr, *iz = nullptr;
+    uint16_t *X = nullptr;
+    void *Y = nullptr;                 // max_batch x rows x 4 bytes
+    cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;
+    static constexpr int kSlots = 64;
+    cudaEvent_t ev_in[kSlots] = {}, ev_run[kSlots] = {};
+};
+
+static void layer_free(lrbi_layer *L)
+{
+    if (!L) return;
+    cudaFree(L->W); cudaFree(L->ip); cudaFree(L->iz); cudaFree(L->X); cudaFree(L->Y);
+    for (int i = 0; i < lrbi_layer::kSlots; ++i) {
+        if (L->ev_in[i]) cudaEventDestroy(L->ev_in[i]);
+        if (L->ev_run[i]) cudaEventDestroy(L->ev_run[i]);
+    }
+    if (L->s_in) cudaStreamDestroy(L->s_in);
+    if (L->s_run) cudaStreamDestroy(L->s_run);
+    if (L->s_out) cudaStreamDestroy(L->s_out);
+    delete L;
+}
+
+lrbi_status lrbi_layer_create(const lrbi_layout *layout, const uint16_t *W_host, const uint32_t *ip_host,
+                              const uint32_t *iz_host, int32_t max_batch, lrbi_layer **out)
+{
+    if (!layout_ok(layout) || !W_host || !ip_host || !iz_host || !out || max_batch < 1) return LRBI_ERR_INVALID_ARG;
+    lrbi_layer *L = new (std::nothrow) lrbi_layer;
+    if (!L) return LRBI_ERR_CUDA;
+    L->layout = *layout;
+    L->g = make_geo(*layout);
+    L->max_batch = max_batch;
+    const size_t wb = (size_t)layout->rows * layout->cols * 2;
+    const size_t ipb = lrbi_packed_ip_words(layout) * 4, izb = lrbi_packed_iz_words(layout) * 4;
+    cudaError_t e = cudaSuccess;
+    auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+    step(cudaMalloc(&L->W, wb));
+    step(cudaMalloc(&L->ip, ipb));
+    step(cudaMalloc(&L->iz, izb));
+    step(cudaMalloc(&L->X, (size_t)max_batch * layout->cols * 2));
+    step(cudaMalloc(&L->Y, (size_t)max_batch * layout->rows * 4));
+    step(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
+    step(cudaStreamCreateWithFlags(&L->s_run, cudaStreamNonBlocking));
+    step(cudaStreamCreateWithFlags(&L->s_out, cudaStreamNonBlocking));
+    for (int i = 0; i < lrbi_layer::kSlots; ++i) {
+        step(cudaEventCreateWithFlags(&L->ev_in[i], cudaEventDisableTiming));
+        step(cudaEventCreateWithFlags(&L->ev_run[i], cudaEventDisableTiming));
+    }
+    if (e == cudaSuccess) {
+        step(cudaMemcpy(L->W, W_host, wb, cudaMemcpyHostToDevice));
+        step(cudaMemcpy(L->ip, ip_host, ipb, cudaMemcpyHostToDevice));
+        step(cudaMemcpy(L->iz, iz_host, izb, cudaMemcpyHostToDevice));
+    }
+    if (e != cudaSuccess) { note_cuda_error((int)e); layer_free(L); return LRBI_ERR_CUDA; }
+    *out = L;
+    return LRBI_OK;
+}
+
+lrbi_status lrbi_layer_forward_host(lrbi_layer *L, const uint16_t *X_host, int32_t batch, void *Y_host,
+                                    int32_t y_dtype, int32_t algo)
+{
+    if (!L || !X_host || !Y_host || batch < 1 || batch > L->max_batch) return LRBI_ERR_INVALID_ARG;
+    if (y_dtype != LRBI_Y_BF16 && y_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
+    const int cols = L->layout.cols, rows = L->layout.rows;
+    const size_t ysz = y_dtype == LRBI_Y_F32 ? 4 : 2;
+    // Chunks of the batch flow through three streams: copy in, compute, copy out.  With pinned
+    // host buffers the three overlap; with pageable ones the copies serialise but stay correct.
+    int chunk = batch;
+    if (batch >= 1024) chunk = 512;
+    int nchunks = (batch + chunk - 1) / chunk;
+    if (nchunks > lrbi_layer::kSlots) { chunk = (batch + lrbi_layer::kSlots - 1) / lrbi_layer::kSlots; chunk = (chunk + 255) / 256 * 256; nchunks = (batch + chunk - 1) / chunk; }
+    cudaError_t e = cudaSuccess;
+    auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+    lrbi_status st = LRBI_OK;
+    for (int c = 0; c < nchunks && e == cudaSuccess && st == LRBI_OK; ++c) {
+        const int b0 = c * chunk, nb = (batch - b0 < chunk) ? batch - b0 : chunk;
+        uint16_t *xd = L->X + (size_t)b0 * cols;
+        uint8_t *yd = static_cast<uint8_t *>(L->Y) + (size_t)b0 * rows * ysz;
+        step(cudaMemcpyAsync(xd, X_host + (size_t)b0 * cols, (size_t)nb * cols * 2, cudaMemcpyHostToDevice, L->s_in));
+        step(cudaEventRecord(L->ev_in[c], L->s_in));
+        step(cudaStreamWaitEvent(L->s_run, L->ev_in[c], 0));
+        if (e != cudaSuccess) break;
+        st = lrbi_masked_gemm(&L->layout, L->W, L->ip, L->iz, xd, nb, yd, y_dtype, algo, L->s_run);
+        if (st != LRBI_OK) break;
+        step(cudaEventRecord(L->ev_run[c], L->s_run));
+        step(cudaStreamWaitEvent(L->s_out, L->ev_run[c], 0));
+        step(cudaMemcpyAsync(static_cast<uint8_t *>(Y_host) + (size_t)b0 * rows * ysz, yd, (size_t)nb * rows * ysz,
+                             cudaMemcpyDeviceToHost, L->s_out));
+    }
+    cudaError_t e2 = cudaStreamSynchronize(L->s_in);
+    cudaError_t e3 = cudaStreamSynchronize(L->s_run);
+    cudaError_t e4 = cudaStreamSynchronize(L->s_out);
+    if (e == cudaSuccess) e = e2 != cudaSuccess ? e2 : (e3 != cudaSuccess ? e3 : e4);
+    if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
+    return st;
+}
+
+lrbi_status lrbi_layer_destroy(lrbi_layer *L)
+{
+    if (!L) return LRBI_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    layer_free(L);
+    return LRBI_OK;
+}
+
+}  // extern "C"

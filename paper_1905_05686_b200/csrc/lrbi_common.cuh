@@ -1,0 +1,76 @@
+// Shared declarations of the lrbi CUDA library (device geometry, status word, launch helpers).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lrbi.h"
+
+namespace lrbi {
+
+// Geometry handed to every kernel by value.
+struct Geo {
+    int rows, cols;   // N_out, K_in
+    int tm, tn;       // tile rows / cols
+    int k, kw;        // rank, words per packed row/column
+    int gr, gc;       // tile grid
+    int pitch;        // mask words per row = ceil(cols / 32)
+};
+
+inline Geo make_geo(const lrbi_layout &l)
+{
+    Geo g;
+    g.rows = l.rows; g.cols = l.cols; g.tm = l.tile_rows; g.tn = l.tile_cols;
+    g.k = l.rank; g.kw = (l.rank + 31) / 32;
+    g.gr = (l.rows + l.tile_rows - 1) / l.tile_rows;
+    g.gc = (l.cols + l.tile_cols - 1) / l.tile_cols;
+    g.pitch = (l.cols + 31) / 32;
+    return g;
+}
+
+// Codes a kernel leaves in the device status word when a bounded wait runs out.
+enum : int {
+    DEV_OK = 0,
+    DEV_TIMEOUT_FULL = 0x100,   // MMA issuer waited for a filled stage
+    DEV_TIMEOUT_EMPTY = 0x200,  // a producer waited for a free stage
+    DEV_TIMEOUT_ACCUM = 0x300,  // epilogue waited for the accumulator
+    DEV_TIMEOUT_DRAIN = 0x400   // drain of in-flight bulk copies on the abort path
+};
+
+// Device status word (one per device that loads the module) and the host-side accessors.
+int *device_status_ptr();                  // device address, resolved once per device
+void count_launch(int n = 1);
+void note_cuda_error(int code);
+
+// Last word of a packed k-bit row/column: bits >= k are ignored.
+__host__ __device__ inline uint32_t tail_mask(int k)
+{
+    return (k & 31) ? ((1u << (k & 31)) - 1u) : 0xFFFFFFFFu;
+}
+
+// bf16 helpers on raw bit patterns.
+__device__ __forceinline__ float bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xFFFF0000u); }
+__device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u);  // quiet NaN
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+// Kernel launchers (one translation unit each).
+lrbi_status launch_decode_ballot(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
+lrbi_status launch_decode_planes(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
+bool decode_planes_supported(const Geo &g);
+
+lrbi_status launch_gemm_generic(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                                const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+bool gemv_supported(const Geo &g, int batch);
+lrbi_status launch_gemv(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                        const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+bool gemm_tc_supported(const Geo &g, int batch);
+// `partials` == nullptr lets the launcher use the library-owned buffer when it splits K.
+lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+
+}  // namespace lrbi
