@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the fused decode + masked-GEMM path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole path (fetch the tile factors, Boolean product, prune W, dense
+product, epilogue) over one batch of seeded synthetic activations.  Rank 0 prints ONE JSON line.
+With N > 1 (launched by torch.distributed.run) every rank runs the same layer on its own batch
+(independent batches, no data-path collective): weak scaling, time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1905_05686_b200 import synth  # noqa: E402
+
+METRIC = "fused decode+masked-GEMM TFLOP/s and effective HBM GB/s vs roofline"
+DEFAULT_WORKLOAD = "ffn_16384x4096"
+L2_BYTES = 126 * 1024 * 1024
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def algorithmic_bytes(layer: synth.Layer, batch: int, y_bytes: int = 2) -> int:
+    """Bytes the method itself must move once: W, packed factors, X, Y."""
+    gr, gc = layer.grid
+    idx = gr * gc * (layer.tile_rows + layer.tile_cols) * layer.kw * 4
+    return 2 * layer.rows * layer.cols + idx + 2 * batch * layer.cols + y_bytes * batch * layer.rows
+
+
+def decode_bytes(layer: synth.Layer) -> int:
+    gr, gc = layer.grid
+    return gr * gc * (layer.tile_rows + layer.tile_cols) * layer.kw * 4 + layer.mask_words * 4
+
+
+def dense_flops(layer: synth.Layer, batch: int) -> int:
+    return 2 * batch * layer.rows * layer.cols
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def reduce_max(value: float, dist=None) -> float:
+    """Max of a per-rank timing over all ranks (identity without a process group)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return value
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([value], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank draws its own activations; weights and index are the same layer on every rank."""
+    return base_seed + 1000 * rank
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+def oracle_sample_run(layer: synth.Layer, batch: int, target_s: float = 15.0, rows_sample=None):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: the full index decode
+    of the layer plus the masked product for the first `sb` batch rows.  Returns (flops, seconds, text)."""
+    import oracle
+
+    Ip, Iz = synth.make_factors(layer)
+    Wb = synth.make_weights(layer)
+    Xb = synth.make_activations(layer, batch)
+    t0 = time.perf_counter()
+    M = oracle.decode_mask(Ip, Iz, layer.rows, layer.cols)
+    t_dec = time.perf_counter() - t0
+    if rows_sample is None:
+        t0 = time.perf_counter()
+        oracle.masked_gemm(Wb, M, Xb[:1])
+        t1 = max(time.perf_counter() - t0, 1e-4)
+        rows_sample = int(max(1, min(batch, (target_s - t_dec) / t1)))
+    t0 = time.perf_counter()
+    oracle.masked_gemm(Wb, M, Xb[:rows_sample])
+    t_gemm = time.perf_counter() - t0
+    flops = dense_flops(layer, rows_sample)
+    text = "full index decode (%d x %d) + masked product for the first %d of %d batch rows" % (
+        layer.rows, layer.cols, rows_sample, batch)
+    return flops, t_dec + t_gemm, text, rows_sample
+
+
+def run_reference(args):
+    import oracle
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    layer = synth.CONFIGS[args.workload]
+    batch = args.batch or layer.batches[-1]
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    # one step = one bounded sample; size it so warm-up + steps stay within a few minutes in total
+    per_step = max(2.0, min(15.0, 150.0 / (steps + warmup)))
+    rows_sample = None
+    times = []
+    flops = 0
+    text = ""
+    for i in range(warmup + steps):
+        flops, sec, text, rows_sample = oracle_sample_run(layer, batch, per_step, rows_sample)
+        if i >= warmup:
+            times.append(sec)
+    ms = 1e3 * float(np.mean(times))
+    value = flops / (ms * 1e-3) / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": batch, "rows": layer.rows, "cols": layer.cols,
+                   "tile": [layer.tile_rows, layer.tile_cols], "rank": layer.rank, "density": layer.density},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle", "sample": text},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def time_calls(fn, n, warmup, flush_buf=None, stream=None):
+    """Per-call device times (ms) with CUDA events on the launching stream."""
+    import torch
+
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+    for i in range(n):
+        if flush_buf is not None:
+            flush_buf.add_(1)                      # rewrites a buffer larger than L2 between timed calls
+        starts[i].record()
+        fn()
+        ends[i].record()
+    torch.cuda.synchronize()
+    return [s.elapsed_time(e) for s, e in zip(starts, ends)]
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_1905_05686_b200 import binding as B
+
+    B.lib()
+    peaks = load_peaks()
+    layer = synth.CONFIGS[args.workload]
+    decode_only = not layer.batches
+    batch = 0 if decode_only else (args.batch or layer.batches[-1])
+
+    Ip, Iz = synth.make_factors(layer)
+    ipw, izw = synth.pack_ip(Ip), synth.pack_iz(Iz)
+    ip, iz = B.to_device_words(ipw), B.to_device_words(izw)
+    flush = None
+    if decode_only:
+        out = torch.empty((layer.rows, (layer.cols + 31) // 32), dtype=torch.int32, device="cuda")
+        step = lambda: B.lrbi_decode_mask(layer, ip, iz, out)
+        work_bytes, work_flops = decode_bytes(layer), 0
+    else:
+        Wb = synth.make_weights(layer)
+        xlayer = synth.Layer(**{**layer.__dict__, "seed": rank_seed(layer.seed, rank)})
+        Xb = synth.make_activations(xlayer, batch)
+        W, X = B.to_device_bf16(Wb), B.to_device_bf16(Xb)
+        Y = torch.empty((batch, layer.rows), dtype=torch.bfloat16, device="cuda")
+        step = lambda: B.lrbi_masked_gemm(layer, W, ip, iz, X, Y=Y)
+        work_bytes, work_flops = algorithmic_bytes(layer, batch), dense_flops(layer, batch)
+    footprint = work_bytes
+    if footprint <= L2_BYTES:
+        flush = torch.zeros(256 * 1024 * 1024 // 4, dtype=torch.int32, device="cuda")
+
+    # ---- device-timed region: K steps, barrier + synchronize on both sides, max over ranks
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = B.launch_count()
+    t_wall0 = time.perf_counter()
+    if flush is None:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        ev[0].record()
+        for i in range(args.steps):
+            step()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+        total_ms = ev[0].elapsed_time(ev[-1])
+    else:
+        per_step = time_calls(step, args.steps, 0, flush)
+        total_ms = float(sum(per_step))
+    launches = B.launch_count() - launches0
+    # keep the sampler alive long enough to see the load, then stop it
+    while time.perf_counter() - t_wall0 < 0.6:
+        step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    total_ms = reduce_max(total_ms, dist if world > 1 else None)
+    ms_per_step = total_ms / args.steps
+    if B.device_status() != 0:
+        raise SystemExit("device status word is not clean: %d" % B.device_status())
+
+    unit = "GB/s" if decode_only else "TFLOP/s"
+    if decode_only:
+        value = world * work_bytes / (ms_per_step * 1e-3) / 1e9
+    else:
+        value = world * work_flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end through the host-buffer entry point (pinned host X and Y, copies inside the timing)
+    e2e = None
+    if not decode_only:
+        hl = B.HostLayer(layer, Wb, ipw, izw, batch)
+        Xh = torch.from_numpy(Xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+        Yh = torch.empty((batch, layer.rows), dtype=torch.bfloat16).pin_memory()
+        for _ in range(3):
+            hl.forward_host(Xh, Yh)
+        n_e2e = max(3, min(args.steps, 10))
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            hl.forward_host(Xh, Yh)            # returns when Y_host is complete
+        e2e_ms = 1e3 * (time.perf_counter() - t0) / n_e2e
+        e2e_ms = reduce_max(e2e_ms, dist if world > 1 else None)
+        e2e = {"value": world * work_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2),
+               "api": "lrbi_layer_forward_host (weights and index resident, X and Y in pinned host memory)"}
+        # the host-buffer call works through the batch in chunks, so K may be split differently:
+        # same values up to fp32 summation order and one bf16 rounding
+        y_dev, y_host = Y.float().cpu(), Yh.float()
+        if not (torch.linalg.norm(y_dev - y_host) <= 4e-3 * torch.linalg.norm(y_dev)):
+            raise SystemExit("host-buffer entry point disagrees with the device entry point")
+        hl.close()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel (one launch per step for this workload)
+    launches_per_step = launches / args.steps
+    kernel_ms = float(np.mean(per_step))
+    if decode_only or B.masked_gemm_choice(layer, batch) == B.ALGO_GEMV or work_flops / work_bytes < peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9):
+        achieved = work_bytes / (kernel_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None}
+    else:
+        achieved = work_flops / (kernel_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                    "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
+    roofline["peak_source"] = "of " + peaks["source"]
+    roofline["kernel_ms"] = kernel_ms
+    roofline["launches_per_step"] = launches_per_step
+
+    # ---- CPU oracle on a bounded sample of the same workload
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        if decode_only:
+            t0 = time.perf_counter()
+            oracle.decode_mask(Ip, Iz, layer.rows, layer.cols)
+            sec = time.perf_counter() - t0
+            cpu = {"value": work_bytes / sec / 1e9, "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle",
+                   "sample": "the whole index decode, once", "seconds": sec}
+        else:
+            flops, sec, text, _ = oracle_sample_run(layer, batch, 15.0)
+            cpu = {"value": flops / sec / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                   "sample": text, "seconds": sec}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32" if decode_only else "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": batch, "rows": layer.rows, "cols": layer.cols,
+                   "tile": [layer.tile_rows, layer.tile_cols], "rank": layer.rank, "density": layer.density,
+                   "kernel": "decode" if decode_only else B.ALGO_NAMES[B.masked_gemm_choice(layer, batch)],
+                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between timed calls (256 MiB rewrite)",
+                   "algorithmic_bytes": work_bytes, "dense_flops": work_flops,
+                   "effective_hbm_gbs": work_bytes / (ms_per_step * 1e-3) / 1e9},
+        "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if cpu:
+        line["cpu_baseline"] = cpu
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(synth.CONFIGS))
+    ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 50 and args.warmup == 5:
+            args.steps, args.warmup = 3, 1
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
