@@ -8,19 +8,28 @@
 // block feeds a 128 x BN x 64 MMA: with BN = 256 every decoded index bit is amortised over 256
 // multiply-accumulates, which keeps the integer work of the decode under the MMA time.
 //
-// Warp roles in a 320-thread block:
-//   warp 0      lane 0 issues the TMA loads of X (cp.async.bulk.tensor, 128B swizzle, zero fill
-//               outside the matrix) into the B stages.
+// Warp roles in a 448-thread block:
+//   warp 0      lane 0 issues the TMA loads (cp.async.bulk.tensor, 128B swizzle, zero fill outside
+//               the matrix) of the X tile into the B stage and of the raw W tile into the A stage.
 //   warp 1      allocates tensor memory; lane 0 issues tcgen05.mma for each filled stage and
 //               commits the stage's "empty" barrier; finally commits the accumulator barrier.
-//   warps 2-9   mask producers.  Each thread owns one 16-byte chunk column (8 weights) and four
-//               rows of the 128 x 64 block: it loads W with coalesced 16-byte loads, one K block
-//               ahead, decodes the eight index bits per row from the row words of Ip and the
-//               column words of Iz ((ip & iz) != 0, Eq. 3), zeroes pruned bf16 values and stores
-//               the chunk at its swizzled position in the A stage.  Writes are made visible to
-//               the tensor core with fence.proxy.async before the stage barrier is signalled.
-//               After the last K block the same warps run the epilogue: tcgen05.ld of their
-//               32-lane quadrant, conversion, stores to Y (or fp32 partial sums when K is split).
+//   warps 10-13 index decoders, one panel (PW*32 columns, all inside one tile) ahead of the pruning
+//               warps.  They transpose the panel's column words of Iz into k bit-planes (plane l =
+//               row l of Iz, 32 columns per word; a warp-wide 32x32 bit transpose, i.e. what 32
+//               __ballot_sync votes would give), then each thread ORs, for one of the 128 rows, the
+//               planes selected by the set bits of that row's Ip word.  That is Eq. 3 evaluated 32
+//               columns per bitwise instruction; the result, the decoded index of the 128 x panel
+//               block, stays bit-packed in shared memory (double buffered) and goes nowhere else.
+//   warps 2-9   pruning warps.  A thread owns four 16-byte chunks of one row of the 128 x 64 block.
+//               When the stage's copies have landed it reads its chunks from the A stage, expands
+//               its 32 index bits to bf16 AND-masks (a shift puts four bits on the sign positions of
+//               the four bytes, prmt replicates each sign over a 16-bit half), zeroes pruned
+//               weights and writes the chunks back in place.  The writes are made visible to the
+//               tensor core with fence.proxy.async before the stage's "masked" barrier is signalled.
+//               No pruning warp ever waits on global memory.  After the last K block the same warps
+//               run the epilogue: tcgen05.ld of their 32-lane quadrant, conversion, transposition
+//               through shared memory, and 16-byte row-contiguous stores to Y (or fp32 partial sums
+//               when K is split).
 //
 // Every barrier wait is bounded by a wall-clock limit.  A wait that runs out records a code in
 // the device status word and raises a block-wide abort flag; every role then leaves its loop, the
@@ -31,12 +40,14 @@
 
 namespace lrbi {
 
-constexpr int TC_THREADS = 320;
+constexpr int TC_THREADS = 448;
 constexpr int TC_BM = 128;                 // rows of W per block (MMA M)
 constexpr int TC_BK = 64;                  // columns per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_A_STAGE_BYTES = TC_BM * TC_BK * 2;
-constexpr int TC_MASK_WARPS = 8;
-constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // 2 s
+constexpr int TC_MASK_WARPS = 8;           // warps 2-9: prune the W tile of each stage, then run the epilogue
+constexpr int TC_DECODE_WARPS = 4;         // warps 10-13: decode the index one panel ahead
+constexpr long long TC_WAIT_LIMIT_CYCLES = 4000000000ll;          // about 2 s of SM clock
+constexpr uint32_t TC_SUSPEND_HINT_NS = 20000u;                   // a waiting thread may sleep this long per try
 
 // ------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -58,34 +69,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(TC_SUSPEND_HINT_NS) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
 // Bounded wait.  Returns false if the block is aborting or the limit ran out (then it records
-// `code` and raises the abort flag).
+// `code` and raises the abort flag).  The limit is counted on the SM's own cycle counter, which is
+// cheap to read; it is looked at once every 64 unsuccessful tries.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           int *status, int code)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    int spins = 0;
-    while (true) {
+    long long t0 = 0;
+    unsigned backoff = 32;
+    for (unsigned spins = 1;; ++spins) {
+        // back off between tries: a hot polling loop steals issue slots and shared-memory queue
+        // bandwidth from the warps that are doing the work this warp is waiting for
+        __nanosleep(backoff);
+        if (backoff < 256) backoff <<= 1;
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((++spins & 255) == 0 && global_ns() - t0 > TC_WAIT_LIMIT_NS) {
-            atomicCAS(status, 0, code);
-            *abort_flag = 1;
-            __threadfence_block();
-            return false;
+        if ((spins & 63u) == 0) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > TC_WAIT_LIMIT_CYCLES) {
+                atomicCAS(status, 0, code);
+                *abort_flag = 1;
+                __threadfence_block();
+                return false;
+            }
         }
     }
 }
@@ -150,19 +163,16 @@ __host__ __device__ constexpr uint32_t make_idesc(int bn)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
-__device__ __forceinline__ uint4 ldg_w(const uint16_t *p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-
 // Shared-memory bookkeeping that follows the operand stages.
 struct TcCtl {
-    uint64_t full[8];
-    uint64_t empty[8];
+    uint64_t full[8];        // TMA copies of a stage have landed
+    uint64_t masked[8];      // ... and its W tile has been pruned in place
+    uint64_t empty[8];       // the MMAs that read the stage have completed
     uint64_t accum;
+    uint64_t epi;            // the eight pruning warps meet here before the epilogue's copy-out
+    uint64_t bits_ready[2];  // decoders -> pruners: the index bits of a panel are in buffer b
+    uint64_t bits_free[2];   // pruners -> decoders: buffer b may be overwritten
+    uint64_t dsync;          // the four decoder warps meet here once per panel
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -170,38 +180,96 @@ struct TcCtl {
 // --------------------------------------------------------------------------------------
 // kernel
 // --------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Bit position of column e (0..31) inside a plane / index word.  Column e = 4g + i sits at bit
+// 8i + 7 - g, so that `word << g` leaves the four bits of group g on the sign positions of the
+// four bytes.  column_of_bit is the inverse (which column a ballot lane stands for).
+__device__ __forceinline__ int column_of_bit(int bit) { return 4 * (7 - (bit & 7)) + (bit >> 3); }
+
+// 32 x 32 bit-matrix transpose across a warp: lane L gives the word x_L, lane l receives the word
+// whose bit L is bit l of x_L.  Five butterfly stages of one shuffle each.  It yields the same
+// 32 words as 32 __ballot_sync votes on ((x >> l) & 1), l = 0..31, at a sixth of the instructions.
+__device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane)
+{
+#pragma unroll
+    for (int stage = 0; stage < 5; ++stage) {
+        const int j = 16 >> stage;
+        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
+                         : stage == 3 ? 0x33333333u : 0x55555555u;
+        const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, j);
+        const bool upper = (lane & j) != 0;
+        const uint32_t sh = upper ? (y >> j) : (y << j);
+        const uint32_t keep = upper ? ~m : m;
+        x = (x & keep) | (sh & ~keep);
+    }
+    return x;
+}
+
+// Zero the pruned halves of the eight bf16 values of one 16-byte chunk.  `bits` holds the index
+// bits of the row's 32 columns in the permuted order above; chunk j uses groups 2j and 2j+1.
+__device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
+{
+    const uint32_t t0 = bits << (2 * j), t1 = bits << (2 * j + 1);
+    w.x &= prmt(t0, t0, 0x9988u);       // sign of byte 0 -> low half, sign of byte 1 -> high half
+    w.y &= prmt(t0, t0, 0xBBAAu);       // bytes 2 and 3
+    w.z &= prmt(t1, t1, 0x9988u);
+    w.w &= prmt(t1, t1, 0xBBAAu);
+    return w;
+}
+
 // grid = (batch tiles, row tiles of 128, K splits).  When gridDim.z > 1 the block writes fp32
 // partial sums to `partials` [split][batch][rows]; a second kernel adds them up.
-template <int BN, int KW>
+// PW = 32-bit index words per row of a panel (8: 256-column panels, 2: 64-column panels).
+template <int BN, int PW>
 __global__ void __launch_bounds__(TC_THREADS)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, Geo g, const uint16_t *__restrict__ W,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
                int stages, int *status)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    extern __shared__ __align__(1024) uint8_t smem[];    // swizzled operand stages need 1024-byte alignment
     constexpr int B_STAGE_BYTES = BN * TC_BK * 2;
     constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    constexpr int KBP = PW / 2;                          // K blocks per panel
+    constexpr int PWH = PW / 2;                          // index words a thread decodes per row
     uint8_t *a_base = smem;
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
-    TcCtl *ctl = reinterpret_cast<TcCtl *>(b_base + (size_t)stages * B_STAGE_BYTES);
+    uint32_t *row_bits = reinterpret_cast<uint32_t *>(b_base + (size_t)stages * B_STAGE_BYTES);   // [2][128][PW]
+    uint32_t *planes = row_bits + 2 * TC_BM * PW;                                                  // [2][kw*32][PW]
+    TcCtl *ctl = reinterpret_cast<TcCtl *>(planes + 2 * g.kw * 32 * PW);
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((smem_u32(smem) & 1023u) != 0) {                 // never expected; refuse rather than compute garbage
+        if (threadIdx.x == 0) atomicCAS(status, 0, DEV_BAD_SMEM_ALIGN);
+        return;
+    }
     const int b0 = blockIdx.x * BN;                      // first batch row of this block
     const int o0 = blockIdx.y * TC_BM;                   // first row of W of this block
     const int nkb_total = (g.cols + TC_BK - 1) / TC_BK;
-    const int kb_begin = blockIdx.z * kb_per_split;
+    const int kb_begin = blockIdx.z * kb_per_split;      // a multiple of KBP
     const int kb_end = min(nkb_total, kb_begin + kb_per_split);
     const int nkb = kb_end - kb_begin;                   // >= 1 by construction of the grid
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
-            mbar_init(&ctl->full[s], 1 + TC_MASK_WARPS);
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->masked[s], TC_MASK_WARPS);
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum, 1);
+        mbar_init(&ctl->epi, TC_MASK_WARPS);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&ctl->bits_ready[b], TC_DECODE_WARPS);
+            mbar_init(&ctl->bits_free[b], TC_MASK_WARPS);
+        }
+        mbar_init(&ctl->dsync, TC_DECODE_WARPS);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -214,20 +282,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, Geo g, const uint16_t 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer (X tiles)
         if (lane == 0) {
-            int armed = 0;
+            bool issued = false;
+            int s = 0;
+            uint32_t parity = 1;                        // a fresh barrier reports its "previous" phase complete
             for (int it = 0; it < nkb; ++it) {
-                const int s = it % stages, round = it / stages;
-                if (round > 0 && !mbar_wait(&ctl->empty[s], (round - 1) & 1, abort_flag, status, DEV_TIMEOUT_EMPTY)) break;
-                mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES);
-                tma_load_2d(b_base + (size_t)s * B_STAGE_BYTES, &x_map, &ctl->full[s], (kb_begin + it) * TC_BK, b0);
-                armed = it + 1;
+                if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) break;
+                mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES + TC_A_STAGE_BYTES);
+                tma_load_2d(a_base + s * TC_A_STAGE_BYTES, &w_map, &ctl->full[s], (kb_begin + it) * TC_BK, o0);
+                tma_load_2d(b_base + s * B_STAGE_BYTES, &x_map, &ctl->full[s], (kb_begin + it) * TC_BK, b0);
+                issued = true;
+                if (++s == stages) { s = 0; parity ^= 1; }
             }
-            if (*abort_flag) {
-                // drain: copies already issued must land before this block's shared memory goes away.
-                // A full barrier also needs the mask warps' arrivals, which may never come now, so
-                // the wait is on elapsed time only (bounded), long enough for any copy in flight.
-                const unsigned long long t0 = global_ns();
-                while (armed > 0 && global_ns() - t0 < 2000000ull) { }
+            if (*abort_flag && issued) {
+                // Abort path: copies already issued must land before this block's shared memory is
+                // given up.  Wait on elapsed cycles alone (bounded): about 2 ms, far beyond any copy
+                // in flight.
+                const long long t0 = clock64();
+                while (clock64() - t0 < 4000000ll) { }
             }
         }
     } else if (warp == 1) {
@@ -235,150 +306,252 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, Geo g, const uint16_t 
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(BN);
             bool ok = true;
+            int s = 0;
+            uint32_t parity = 0;
             for (int it = 0; it < nkb && ok; ++it) {
-                const int s = it % stages, round = it / stages;
-                ok = mbar_wait(&ctl->full[s], round & 1, abort_flag, status, DEV_TIMEOUT_FULL);
+                ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t da = make_sw128_desc(smem_u32(a_base + (size_t)s * TC_A_STAGE_BYTES));
-                const uint64_t db = make_sw128_desc(smem_u32(b_base + (size_t)s * B_STAGE_BYTES));
+                const uint64_t da = make_sw128_desc(smem_u32(a_base + s * TC_A_STAGE_BYTES));
+                const uint64_t db = make_sw128_desc(smem_u32(b_base + s * B_STAGE_BYTES));
 #pragma unroll
                 for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
                     // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in address units
                     umma_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
                 }
                 umma_commit(&ctl->empty[s]);            // frees the stage when these MMAs have read it
+                if (++s == stages) { s = 0; parity ^= 1; }
             }
             if (ok) umma_commit(&ctl->accum);           // accumulator complete
         }
-    } else {
-        // ------------------------------------------------------------- mask producers
-        const int mt = threadIdx.x - 64;                // 0..255
-        const int cc = mt & 7;                          // 16-byte chunk column inside the 128-byte row
-        const int rb = mt >> 3;                         // rows rb, rb+32, rb+64, rb+96
+    } else if (warp >= 2 + TC_MASK_WARPS) {
+        // ------------------------------------------------------------- index decoders
+        const int dt = threadIdx.x - (2 + TC_MASK_WARPS) * 32;   // 0..127: row of the block this thread decodes
+        const int dw = dt >> 5;                         // decoder warp 0..3
         const uint32_t tail = tail_mask(g.k);
         const int tr = o0 / g.tm;                       // the 128 rows lie in one tile row
-        const int i0 = o0 - tr * g.tm;
+        const int i_row = o0 - tr * g.tm + dt;          // row inside the tile
+        const bool row_ok = o0 + dt < g.rows && i_row < g.tm;
+        const int bit_col = column_of_bit(lane);        // column (0..31) this lane stands for in a transpose
+        const int npairs = g.kw * PW;                   // (32-plane block, index word) pairs of a panel
+        const int npanels = (nkb + KBP - 1) / KBP;
+        constexpr int ZREG = 4, XREG = 2;               // factor words kept in registers one panel ahead
+        const bool pre = npairs <= ZREG * TC_DECODE_WARPS && g.kw <= XREG;   // true for k <= 64
 
-        uint32_t ipv[4][KW];
-        int tc_prev = -1;
-        uint4 wnext[4];
-        uint4 znext[2 * KW];
-
-        auto fetch = [&](int it, uint4 (&wv)[4], uint4 (&zv)[2 * KW]) {
-            const int c = (kb_begin + it) * TC_BK + cc * 8;          // first of this thread's 8 columns
-            const bool colok = it < nkb && c < g.cols;
+        struct PanelAt { const uint32_t *iz_tile; const uint32_t *ip_row; int c0; int j0; bool live; };
+        auto panel_at = [&](int P) {
+            PanelAt p;
+            p.live = P < npanels;
+            p.c0 = (kb_begin + P * KBP) * TC_BK;        // first column of the panel
+            const int tc = p.live ? p.c0 / g.tn : 0;
+            p.j0 = p.c0 - tc * g.tn;                    // ... inside its tile
+            const size_t tile = (size_t)tr * g.gc + tc;
+            p.iz_tile = iz + tile * g.tn * g.kw;
+            p.ip_row = ip + (tile * g.tm + (row_ok ? i_row : 0)) * g.kw;
+            return p;
+        };
+        auto load_z = [&](const PanelAt &p, int n) -> uint32_t {     // column word of pair dw + 4n, this lane's column
+            const int pi = dw + TC_DECODE_WARPS * n;
+            if (!p.live || pi >= npairs) return 0u;
+            const int lb = pi / PW, off = (pi % PW) * 32 + bit_col;
+            uint32_t z = 0;
+            if (p.c0 + off < g.cols && p.j0 + off < g.tn) z = __ldg(p.iz_tile + (p.j0 + off) * g.kw + lb);
+            return (lb == g.kw - 1) ? (z & tail) : z;
+        };
+        auto load_ip = [&](const PanelAt &p, int lb) -> uint32_t {   // row word lb of this thread's row
+            if (!p.live || !row_ok || lb >= g.kw) return 0u;
+            const uint32_t x = __ldg(p.ip_row + lb);
+            return (lb == g.kw - 1) ? (x & tail) : x;
+        };
+        // statically indexed only (fully unrolled loops): they stay in registers while loads are in flight
+        uint32_t zreg[ZREG], xreg[XREG];
+        {
+            const PanelAt p0 = panel_at(0);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int o = o0 + rb + 32 * q;
-                wv[q] = (colok && o < g.rows) ? ldg_w(W + (long long)o * g.cols + c) : make_uint4(0, 0, 0, 0);
+            for (int n = 0; n < ZREG; ++n) zreg[n] = pre ? load_z(p0, n) : 0u;
+#pragma unroll
+            for (int lb = 0; lb < XREG; ++lb) xreg[lb] = pre ? load_ip(p0, lb) : 0u;
+        }
+        uint32_t dsync_parity = 0;
+        bool ok = true;
+        for (int P = 0; P < npanels && ok; ++P) {
+            const int buf = P & 1;
+            uint32_t *pl_buf = planes + buf * (g.kw * 32 * PW);
+            uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
+            // the pruning warps must be done with the panel that used this buffer two panels ago
+            ok = mbar_wait(&ctl->bits_free[buf], ((P >> 1) & 1) ^ 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
+            if (!ok) break;
+            // (a) bit-planes of Iz: each lane brings the k-bit word of one column, a warp-wide
+            //     transpose turns 32 column words into 32 plane words (lane l keeps plane lb*32 + l)
+            const PanelAt pc = panel_at(P), pn = panel_at(P + 1);
+            uint32_t xcur[XREG];
+            if (pre) {
+#pragma unroll
+                for (int n = 0; n < ZREG; ++n) {
+                    const int pi = dw + TC_DECODE_WARPS * n;
+                    if (pi < npairs) pl_buf[((pi / PW) * 32 + lane) * PW + (pi % PW)] = transpose32(zreg[n], lane);
+                }
+#pragma unroll
+                for (int lb = 0; lb < XREG; ++lb) xcur[lb] = xreg[lb];
+                // next panel's factor words start their trip now
+#pragma unroll
+                for (int n = 0; n < ZREG; ++n) zreg[n] = load_z(pn, n);
+#pragma unroll
+                for (int lb = 0; lb < XREG; ++lb) xreg[lb] = load_ip(pn, lb);
+            } else {
+                for (int n = 0; dw + TC_DECODE_WARPS * n < npairs; ++n) {
+                    const int pi = dw + TC_DECODE_WARPS * n;
+                    pl_buf[((pi / PW) * 32 + lane) * PW + (pi % PW)] = transpose32(load_z(pc, n), lane);
+                }
             }
-            if (colok) {
-                const int tc = c / g.tn, j = c - tc * g.tn;
-                const uint4 *zp = reinterpret_cast<const uint4 *>(iz + (((long long)tr * g.gc + tc) * g.tn + j) * KW);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->dsync);
+            ok = mbar_wait(&ctl->dsync, dsync_parity, abort_flag, status, DEV_TIMEOUT_EMPTY);
+            dsync_parity ^= 1;
+            if (!ok) break;
+            // (b) Eq. 3 for one row: OR of the planes its Ip bits select
+            uint32_t acc[PW];
 #pragma unroll
-                for (int v = 0; v < 2 * KW; ++v) zv[v] = __ldg(zp + v);
+            for (int q = 0; q < PW; ++q) acc[q] = 0;
+            auto or_planes = [&](uint32_t x, int lb) {
+                while (x) {
+                    const int l = lb * 32 + __ffs(x) - 1;
+                    x &= x - 1;
+                    const uint32_t *src = pl_buf + l * PW;
+                    if (PW == 8) {
+                        const uint4 v0 = reinterpret_cast<const uint4 *>(src)[0], v1 = reinterpret_cast<const uint4 *>(src)[1];
+                        acc[0] |= v0.x; acc[1] |= v0.y; acc[2 % PW] |= v0.z; acc[3 % PW] |= v0.w;
+                        acc[4 % PW] |= v1.x; acc[5 % PW] |= v1.y; acc[6 % PW] |= v1.z; acc[7 % PW] |= v1.w;
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < PW; ++q) acc[q] |= src[q];
+                    }
+                }
+            };
+            if (pre) {
+#pragma unroll
+                for (int lb = 0; lb < XREG; ++lb) or_planes(xcur[lb], lb);
+            } else {
+                for (int lb = 0; lb < g.kw; ++lb) or_planes(load_ip(pc, lb), lb);
+            }
+            if (PW == 8) {
+                reinterpret_cast<uint4 *>(rb_buf + dt * PW)[0] = make_uint4(acc[0], acc[1], acc[2 % PW], acc[3 % PW]);
+                reinterpret_cast<uint4 *>(rb_buf + dt * PW)[1] = make_uint4(acc[4 % PW], acc[5 % PW], acc[6 % PW], acc[7 % PW]);
             } else {
 #pragma unroll
-                for (int v = 0; v < 2 * KW; ++v) zv[v] = make_uint4(0, 0, 0, 0);
+                for (int q = 0; q < PW; ++q) rb_buf[dt * PW + q] = acc[q];
             }
-        };
-        fetch(0, wnext, znext);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->bits_ready[buf]);
+        }
+    } else {
+        // ------------------------------------------------------------- pruning warps
+        const int mt = threadIdx.x - 64;                // 0..255
+        const int mw = mt >> 5;                         // pruning warp 0..7
+        // Two lanes share a row: lane pair p of a warp owns row 8*(p/8) + 2*(p%4) + (p/4)%2 of the
+        // warp's 16 rows (so the eight lanes of one store phase fall on eight different swizzled
+        // chunk positions), and lane h of the pair owns the 16-byte chunks h, h+2, h+4, h+6 of the
+        // row's 128 bytes.
+        const int pr = lane >> 1;
+        const int r = mw * 16 + 8 * (pr >> 3) + 2 * (pr & 3) + ((pr >> 2) & 1);   // row of the 128-row block
+        const int h = lane & 1;
+        uint32_t epi_parity = 0;
 
         bool ok = true;
+        int s = 0;                                       // stage of the current K block
+        uint32_t full_parity = 0;
+        int kp = 0;                                      // K block inside its panel
+        int P = 0;                                       // panel index inside this block's K range
         for (int it = 0; it < nkb && ok; ++it) {
-            const int s = it % stages, round = it / stages;
-            uint4 wcur[4], zcur[2 * KW];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) wcur[q] = wnext[q];
-#pragma unroll
-            for (int v = 0; v < 2 * KW; ++v) zcur[v] = znext[v];
-            fetch(it + 1, wnext, znext);                 // next K block in flight while this one is masked
-
-            const int c = (kb_begin + it) * TC_BK + cc * 8;
-            const int tc = min(c, g.cols - 1) / g.tn;
-            if (tc != tc_prev) {                         // row words of Ip change with the tile column
-                tc_prev = tc;
-                const long long tile = (long long)tr * g.gc + tc;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int i = i0 + rb + 32 * q;
-#pragma unroll
-                    for (int w = 0; w < KW; ++w) {
-                        uint32_t v = (i < g.tm) ? __ldg(ip + (tile * g.tm + i) * KW + w) : 0u;
-                        if (w == KW - 1) v &= tail;
-                        ipv[q][w] = v;
-                    }
-                }
+            const int buf = P & 1;
+            if (kp == 0) {                               // first K block of a panel: its index bits must be there
+                ok = mbar_wait(&ctl->bits_ready[buf], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
+                if (!ok) break;
             }
-            uint32_t izv[8][KW];
-#pragma unroll
-            for (int v = 0; v < 2 * KW; ++v) {
-                const uint32_t zz[4] = {zcur[v].x, zcur[v].y, zcur[v].z, zcur[v].w};
-#pragma unroll
-                for (int t = 0; t < 4; ++t) izv[(v * 4 + t) / KW][(v * 4 + t) % KW] = zz[t];
+            const uint2 bits = *reinterpret_cast<const uint2 *>(row_bits + buf * (TC_BM * PW) + r * PW + kp * 2);
+            if (kp == KBP - 1 || it == nkb - 1) {        // last use of this buffer: hand it back to the decoders
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->bits_free[buf]);
             }
-
-            if (round > 0) ok = mbar_wait(&ctl->empty[s], (round - 1) & 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
+            // ---------------- prune 32 weights of one row of the A stage, in place
+            ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
             if (!ok) break;
-
-            uint8_t *a_stage = a_base + (size_t)s * TC_A_STAGE_BYTES;
+            uint8_t *a_row = a_base + s * TC_A_STAGE_BYTES + r * 128;
+            uint4 wv[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int r = rb + 32 * q;
-                uint32_t ww[4] = {wcur[q].x, wcur[q].y, wcur[q].z, wcur[q].w};
+            for (int j = 0; j < 4; ++j) {
+                // 128-byte swizzle: 16-byte chunk c of row r lives at chunk position c ^ (r % 8)
+                const int chunk = 2 * j + h;
+                wv[j] = *reinterpret_cast<const uint4 *>(a_row + ((chunk ^ (r & 7)) << 4));
+            }
 #pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    uint32_t lo = 0, hi = 0;
-#pragma unroll
-                    for (int w = 0; w < KW; ++w) {
-                        lo |= ipv[q][w] & izv[2 * h][w];
-                        hi |= ipv[q][w] & izv[2 * h + 1][w];
-                    }
-                    const uint32_t keep = (lo ? 0x0000FFFFu : 0u) | (hi ? 0xFFFF0000u : 0u);
-                    ww[h] &= keep;                       // pruned weights become +0
-                }
-                // 128-byte swizzle: 16-byte chunk cc of row r lives at chunk position cc ^ (r % 8)
-                uint4 *dst = reinterpret_cast<uint4 *>(a_stage + r * 128 + ((cc ^ (r & 7)) << 4));
-                *dst = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+            for (int j = 0; j < 4; ++j) {                // chunk 2j+h: word (2j+h)/4, chunk-in-word (2j+h)%4
+                const int chunk = 2 * j + h;
+                wv[j] = prune_chunk(wv[j], (j < 2) ? bits.x : bits.y, chunk & 3);
+                *reinterpret_cast<uint4 *>(a_row + ((chunk ^ (r & 7)) << 4)) = wv[j];
             }
             fence_async_proxy();                         // generic-proxy stores -> visible to the MMA
             __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->full[s]);
+            if (lane == 0) mbar_arrive(&ctl->masked[s]);
+            if (++s == stages) { s = 0; full_parity ^= 1; }
+            if (++kp == KBP) { kp = 0; ++P; }
         }
 
         // ------------------------------------------------------------- epilogue (same warps)
         if (ok) ok = mbar_wait(&ctl->accum, 0, abort_flag, status, DEV_TIMEOUT_ACCUM);
         if (ok) {
             tc_fence_after();
+            // All MMAs have completed, so the operand stages are free: reuse them to transpose the
+            // accumulator (lane = output feature) into rows of Y (contiguous output features).
+            const bool out32 = partials != nullptr || y_dtype == LRBI_Y_F32;
             const int quad = warp & 3;                   // tensor-memory lanes this warp may read
-            const int half = (warp - 2) >> 2;            // which half of the accumulator columns
-            const int o = o0 + quad * 32 + lane;
+            const int half = mw >> 2;                    // which half of the accumulator columns
+            const int ol = quad * 32 + lane;             // output feature inside the block
             constexpr int COLS_PER_WARP = BN / 2 < 16 ? 16 : BN / 2;
             constexpr int NCHUNK = COLS_PER_WARP / 16;
-            const bool active = (BN >= 32) || half == 0;
-            if (active) {
+            if ((BN >= 32) || half == 0) {
 #pragma unroll 1
                 for (int ch = 0; ch < NCHUNK; ++ch) {
                     const int col0 = half * COLS_PER_WARP + ch * 16;
                     uint32_t v[16];
                     tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)col0, v);
                     tmem_ld_wait();
-                    if (o < g.rows) {
+                    if (out32) {
+                        float *st = reinterpret_cast<float *>(smem);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int b = b0 + col0 + j;
-                            if (b < batch) {
-                                const float f = __uint_as_float(v[j]);
-                                if (partials) {
-                                    partials[((long long)blockIdx.z * batch + b) * g.rows + o] = f;
-                                } else if (y_dtype == LRBI_Y_F32) {
-                                    reinterpret_cast<float *>(Y)[(long long)b * g.rows + o] = f;
-                                } else {
-                                    reinterpret_cast<uint16_t *>(Y)[(long long)b * g.rows + o] = f32_to_bf16_rne(f);
-                                }
-                            }
-                        }
+                        for (int j = 0; j < 16; ++j) st[(col0 + j) * TC_BM + ol] = __uint_as_float(v[j]);
+                    } else {
+                        uint16_t *st = reinterpret_cast<uint16_t *>(smem);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) st[(col0 + j) * TC_BM + ol] = f32_to_bf16_rne(__uint_as_float(v[j]));
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->epi);
+            ok = mbar_wait(&ctl->epi, epi_parity, abort_flag, status, DEV_TIMEOUT_ACCUM);
+            epi_parity ^= 1;
+            if (ok) {
+                const int esz = out32 ? 4 : 2;
+                uint8_t *dst_base = partials ? reinterpret_cast<uint8_t *>(partials + (long long)blockIdx.z * batch * g.rows)
+                                             : reinterpret_cast<uint8_t *>(Y);
+                const int row_bytes = TC_BM * esz;                       // one batch row of the block
+                const int chunks = row_bytes / 16;                       // 16 (bf16) or 32 (fp32)
+                const int per16 = 16 / esz;                              // outputs per 16-byte chunk
+                const int nb = min(BN, batch - b0);
+                const bool vec_ok = (g.rows % per16) == 0;               // rows of Y stay 16-byte aligned
+                for (int idx = mt; idx < nb * chunks; idx += TC_MASK_WARPS * 32) {
+                    const int bl = idx / chunks, cj = idx - bl * chunks;
+                    const int oc = o0 + cj * per16;                      // first output feature of the chunk
+                    if (oc >= g.rows) continue;
+                    const uint8_t *src = smem + (size_t)bl * row_bytes + cj * 16;
+                    uint8_t *dst = dst_base + ((long long)(b0 + bl) * g.rows + oc) * esz;
+                    if (vec_ok && oc + per16 <= g.rows) {
+                        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+                    } else {
+                        const int n = min(per16, g.rows - oc);
+                        for (int e = 0; e < n * esz; e += 2)
+                            *reinterpret_cast<uint16_t *>(dst + e) = *reinterpret_cast<const uint16_t *>(src + e);
                     }
                 }
             }
@@ -425,14 +598,19 @@ static EncodeTiledFn get_encode_fn()
     return fn;
 }
 
+constexpr int TC_MAX_RANK = 256;
+
 bool gemm_tc_supported(const Geo &g, int batch)
 {
-    if (batch < 1 || g.kw > 2) return false;
+    if (batch < 1 || g.k > TC_MAX_RANK) return false;
     if ((g.cols % 8) != 0) return false;                                   // 16-byte rows for TMA and vector loads
     if (!(g.gr == 1 || (g.tm % TC_BM) == 0)) return false;                 // 128 rows inside one tile row
-    if (!(g.gc == 1 ? (g.tn % 8) == 0 : (g.tn % TC_BK) == 0)) return false; // a K block inside one tile column
+    if (!(g.gc == 1 || (g.tn % TC_BK) == 0)) return false;                 // a K block inside one tile column
     return true;
 }
+
+// Index words per panel row: 256-column panels when every panel then lies inside one tile.
+static int panel_words(const Geo &g) { return (g.gc == 1 || (g.tn % 256) == 0) ? 8 : 2; }
 
 struct Workspace {
     float *ptr = nullptr;
@@ -454,7 +632,7 @@ static float *workspace(size_t bytes)
     return w.ptr;
 }
 
-template <int BN, int KW>
+template <int BN, int PW>
 static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                              const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count)
 {
@@ -469,6 +647,13 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
+    CUtensorMap wmap;
+    const cuuint64_t wdims[2] = {(cuuint64_t)g.cols, (cuuint64_t)g.rows};
+    const cuuint32_t wbox[2] = {TC_BK, TC_BM};
+    r = encode(&wmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(W), wdims, strides, wbox, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
     constexpr int B_STAGE = BN * TC_BK * 2;
     const int nkb = (g.cols + TC_BK - 1) / TC_BK;
@@ -481,27 +666,28 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
         if (splits > 32) splits = 32;
     }
     int kb_per_split = (nkb + splits - 1) / splits;
+    kb_per_split = (kb_per_split + 3) / 4 * 4;                               // splits start on panel boundaries
     splits = (nkb + kb_per_split - 1) / kb_per_split;                        // no empty split
 
     int stages = BN >= 256 ? 4 : (BN >= 128 ? 4 : 6);
     if (stages > 8) stages = 8;
-    const size_t smem = 1024 + (size_t)stages * (TC_A_STAGE_BYTES + B_STAGE) + sizeof(TcCtl);
+    const size_t smem = 1024 + (size_t)stages * (TC_A_STAGE_BYTES + B_STAGE) + (size_t)2 * (TC_BM + g.kw * 32) * PW * 4 + sizeof(TcCtl);
 
     float *partials = nullptr;
     if (splits > 1) {
         partials = workspace((size_t)splits * batch * g.rows * sizeof(float));
         if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
     }
-    auto kern = gemm_tc_kernel<BN, KW>;
+    auto kern = gemm_tc_kernel<BN, PW>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
         attr_done = true;
     }
     dim3 grid((unsigned)((batch + BN - 1) / BN), (unsigned)((g.rows + TC_BM - 1) / TC_BM), (unsigned)splits);
     if (grid.y > 65535 || grid.z > 65535) return LRBI_ERR_UNSUPPORTED;
-    kern<<<grid, TC_THREADS, smem, s>>>(map, g, W, ip, iz, batch, Y, y_dtype, partials, kb_per_split, stages,
+    kern<<<grid, TC_THREADS, smem, s>>>(map, wmap, g, ip, iz, batch, Y, y_dtype, partials, kb_per_split, stages,
                                          device_status_ptr());
     count_launch();
     cudaError_t e = cudaGetLastError();
@@ -520,8 +706,8 @@ template <int BN>
 static lrbi_status launch_tc_kw(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                                 const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count)
 {
-    return g.kw == 1 ? launch_tc<BN, 1>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
-                     : launch_tc<BN, 2>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    return panel_words(g) == 8 ? launch_tc<BN, 8>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
+                               : launch_tc<BN, 2>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
 }
 
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,

@@ -33,7 +33,8 @@ enum : int {
     DEV_TIMEOUT_FULL = 0x100,   // MMA issuer waited for a filled stage
     DEV_TIMEOUT_EMPTY = 0x200,  // a producer waited for a free stage
     DEV_TIMEOUT_ACCUM = 0x300,  // epilogue waited for the accumulator
-    DEV_TIMEOUT_DRAIN = 0x400   // drain of in-flight bulk copies on the abort path
+    DEV_TIMEOUT_DRAIN = 0x400,  // drain of in-flight bulk copies on the abort path
+    DEV_BAD_SMEM_ALIGN = 0x500  // dynamic shared memory did not start on a 1024-byte boundary
 };
 
 // Device status word (one per device that loads the module) and the host-side accessors.

@@ -123,6 +123,9 @@ TC_SHAPES = [
     (256, 2304, 128, 256, 16, 700),
     (1152, 1024, 128, 512, 32, 300),
     (1024, 4096, 512, 1024, 64, 520),
+    (256, 1024, 128, 256, 145, 64),      # the paper's LSTM rank: five index words per row
+    (384, 776, 384, 776, 256, 40),       # one tile, rank 256, ragged last K block
+    (256, 640, 128, 128, 16, 260),       # 128-column tiles: 64-column panels
 ]
 
 
