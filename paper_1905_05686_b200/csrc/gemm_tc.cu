@@ -69,7 +69,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(TC_SUSPEND_HINT_NS) : "memory");
     return ok != 0;
@@ -135,6 +135,50 @@ __device__ __forceinline__ void umma_commit(uint64_t *bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// ---- CTA-pair (cta_group::2) variants: one MMA spans the tensor cores and shared memory of two
+// CTAs of a cluster; the accumulator rows are split between their tensor memories.
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t *dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done.
+__device__ __forceinline__ void umma2_commit_both(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+// Arrive on the barrier at the same offset in the shared memory of CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_remote(uint64_t *bar, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 {
     asm volatile(
@@ -158,15 +202,16 @@ __device__ __forceinline__ uint64_t make_sw128_desc(uint32_t saddr)
     return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = bn.
-__host__ __device__ constexpr uint32_t make_idesc(int bn)
+__host__ __device__ constexpr uint32_t make_idesc(int bn, int m = TC_BM)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // Shared-memory bookkeeping that follows the operand stages.
 struct TcCtl {
     uint64_t full[8];        // TMA copies of a stage have landed
     uint64_t masked[8];      // ... and its W tile has been pruned in place
+    uint64_t peer_masked[8]; // pair mode, leader CTA: the other CTA's stage is pruned too
     uint64_t empty[8];       // the MMAs that read the stage have completed
     uint64_t accum;
     uint64_t epi;            // the eight pruning warps meet here before the epilogue's copy-out
@@ -211,6 +256,35 @@ __device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane)
     return x;
 }
 
+// Four independent transposes with their shuffles interleaved (latency of one, work of four).
+__device__ __forceinline__ void transpose32_x4(uint32_t (&x)[4], int lane)
+{
+#pragma unroll
+    for (int stage = 0; stage < 5; ++stage) {
+        const int j = 16 >> stage;
+        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
+                         : stage == 3 ? 0x33333333u : 0x55555555u;
+        const bool upper = (lane & j) != 0;
+        const uint32_t keep = upper ? ~m : m;
+        uint32_t y[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) y[t] = __shfl_xor_sync(0xFFFFFFFFu, x[t], j);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const uint32_t sh = upper ? (y[t] >> j) : (y[t] << j);
+            x[t] = (x[t] & keep) | (sh & ~keep);
+        }
+    }
+}
+
+// 16-byte asynchronous copy global -> shared; bytes beyond `valid` (0..16) are written as zero.
+__device__ __forceinline__ void cp_async_16(void *dst_smem, const void *src, int valid)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(valid) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 // Zero the pruned halves of the eight bf16 values of one 16-byte chunk.  `bits` holds the index
 // bits of the row's 32 columns in the permuted order above; chunk j uses groups 2j and 2j+1.
 __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
@@ -226,23 +300,34 @@ __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
 // grid = (batch tiles, row tiles of 128, K splits).  When gridDim.z > 1 the block writes fp32
 // partial sums to `partials` [split][batch][rows]; a second kernel adds them up.
 // PW = 32-bit index words per row of a panel (8: 256-column panels, 2: 64-column panels).
-template <int BN, int PW>
-__global__ void __launch_bounds__(TC_THREADS)
+// PAIR: two CTAs of a cluster (neighbours along grid x) share one 256-row x BN-column
+// output tile.  Each loads and prunes its own 128 rows of W and loads its own half of the X tile; the
+// leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2, which reads the operands of both CTAs
+// and leaves each CTA's 128 accumulator rows in its own tensor memory.  Every X tile is then fetched
+// once per 256 rows of W instead of once per 128, and each byte of it is read from shared memory by
+// one tensor core pass instead of two.  Two such blocks are resident per SM (three stages each), so
+// one block's epilogue and panel hand-overs overlap the other's MMAs.
+template <int BN, int PW, bool PAIR>
+__global__ void __launch_bounds__(TC_THREADS, PAIR ? 2 : 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
                int stages, int *status)
 {
     extern __shared__ __align__(1024) uint8_t smem[];    // swizzled operand stages need 1024-byte alignment
-    constexpr int B_STAGE_BYTES = BN * TC_BK * 2;
+    constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // rows of X this CTA loads per stage
+    constexpr int B_STAGE_BYTES = B_ROWS * TC_BK * 2;
     constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
     constexpr int KBP = PW / 2;                          // K blocks per panel
     constexpr int PWH = PW / 2;                          // index words a thread decodes per row
     uint8_t *a_base = smem;
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
+    constexpr int PWS = PW == 8 ? 12 : PW;               // words between planes (padded: conflict-free 16-byte reads)
     uint32_t *row_bits = reinterpret_cast<uint32_t *>(b_base + (size_t)stages * B_STAGE_BYTES);   // [2][128][PW]
-    uint32_t *planes = row_bits + 2 * TC_BM * PW;                                                  // [2][kw*32][PW]
-    TcCtl *ctl = reinterpret_cast<TcCtl *>(planes + 2 * g.kw * 32 * PW);
+    uint32_t *planes = row_bits + 2 * TC_BM * PW;                                                  // [kw*32][PWS]
+    uint32_t *iz_stage = planes + g.kw * 32 * PWS;                                                 // [PW*32][kw]
+    uint32_t *ip_stage = iz_stage + PW * 32 * g.kw;                                                // [128][kw]
+    TcCtl *ctl = reinterpret_cast<TcCtl *>(ip_stage + TC_BM * g.kw);
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -250,8 +335,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         if (threadIdx.x == 0) atomicCAS(status, 0, DEV_BAD_SMEM_ALIGN);
         return;
     }
-    const int b0 = blockIdx.x * BN;                      // first batch row of this block
-    const int o0 = blockIdx.y * TC_BM;                   // first row of W of this block
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u; // 0 = leader of the pair
+    // grid.x runs fastest over blocks that share rows of W, so W streams from HBM once and X stays in L2.
+    // Pair mode: the two CTAs of a cluster are neighbours along x (x = 2 * batch tile + rank), y = 256-row pair.
+    const int b0 = (PAIR ? (blockIdx.x >> 1) : blockIdx.x) * BN;                       // first batch row of the tile
+    const int o0 = (PAIR ? (blockIdx.y * 2 + (int)rank) : blockIdx.y) * TC_BM;          // first row of W of this block
     const int nkb_total = (g.cols + TC_BK - 1) / TC_BK;
     const int kb_begin = blockIdx.z * kb_per_split;      // a multiple of KBP
     const int kb_end = min(nkb_total, kb_begin + kb_per_split);
@@ -261,6 +349,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         for (int s = 0; s < stages; ++s) {
             mbar_init(&ctl->full[s], 1);
             mbar_init(&ctl->masked[s], TC_MASK_WARPS);
+            mbar_init(&ctl->peer_masked[s], 1);
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum, 1);
@@ -273,9 +362,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+    if (warp == 1) {
+        if (PAIR) tmem_alloc2(&ctl->tmem_base, TMEM_COLS);
+        else tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();                        // both CTAs' barriers exist before anyone signals across
     tc_fence_after();
     const uint32_t tmem_d = ctl->tmem_base;
 
@@ -289,7 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) break;
                 mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES + TC_A_STAGE_BYTES);
                 tma_load_2d(a_base + s * TC_A_STAGE_BYTES, &w_map, &ctl->full[s], (kb_begin + it) * TC_BK, o0);
-                tma_load_2d(b_base + s * B_STAGE_BYTES, &x_map, &ctl->full[s], (kb_begin + it) * TC_BK, b0);
+                tma_load_2d(b_base + s * B_STAGE_BYTES, &x_map, &ctl->full[s], (kb_begin + it) * TC_BK, b0 + (int)rank * B_ROWS);
                 issued = true;
                 if (++s == stages) { s = 0; parity ^= 1; }
             }
@@ -303,13 +396,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BN);
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = PAIR ? make_idesc(BN, 2 * TC_BM) : make_idesc(BN);
             bool ok = true;
             int s = 0;
             uint32_t parity = 0;
             for (int it = 0; it < nkb && ok; ++it) {
                 ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
+                if (ok && PAIR) ok = mbar_wait(&ctl->peer_masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t da = make_sw128_desc(smem_u32(a_base + s * TC_A_STAGE_BYTES));
@@ -317,12 +411,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
 #pragma unroll
                 for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
                     // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in address units
-                    umma_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
+                    if (PAIR) umma2_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
+                    else umma_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
                 }
-                umma_commit(&ctl->empty[s]);            // frees the stage when these MMAs have read it
+                // frees the stage (in both CTAs of a pair) when these MMAs have read it
+                if (PAIR) umma2_commit_both(&ctl->empty[s]); else umma_commit(&ctl->empty[s]);
                 if (++s == stages) { s = 0; parity ^= 1; }
             }
-            if (ok) umma_commit(&ctl->accum);           // accumulator complete
+            if (ok) {                                   // accumulator complete
+                if (PAIR) umma2_commit_both(&ctl->accum); else umma_commit(&ctl->accum);
+            }
+        } else if (lane == 0) {
+            // ------------------------------------------------------------- relay (second CTA of a pair)
+            // tells the leader when this CTA's half of a stage is loaded and pruned
+            bool ok = true;
+            int s = 0;
+            uint32_t parity = 0;
+            for (int it = 0; it < nkb && ok; ++it) {
+                ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
+                if (!ok) break;
+                mbar_arrive_remote(&ctl->peer_masked[s], 0);
+                if (++s == stages) { s = 0; parity ^= 1; }
+            }
         }
     } else if (warp >= 2 + TC_MASK_WARPS) {
         // ------------------------------------------------------------- index decoders
@@ -330,94 +440,102 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         const int dw = dt >> 5;                         // decoder warp 0..3
         const uint32_t tail = tail_mask(g.k);
         const int tr = o0 / g.tm;                       // the 128 rows lie in one tile row
-        const int i_row = o0 - tr * g.tm + dt;          // row inside the tile
-        const bool row_ok = o0 + dt < g.rows && i_row < g.tm;
+        const int i0 = o0 - tr * g.tm;                  // first row of the block inside its tile
+        const bool row_ok = o0 + dt < g.rows && i0 + dt < g.tm;
         const int bit_col = column_of_bit(lane);        // column (0..31) this lane stands for in a transpose
         const int npairs = g.kw * PW;                   // (32-plane block, index word) pairs of a panel
         const int npanels = (nkb + KBP - 1) / KBP;
-        constexpr int ZREG = 4, XREG = 2;               // factor words kept in registers one panel ahead
-        const bool pre = npairs <= ZREG * TC_DECODE_WARPS && g.kw <= XREG;   // true for k <= 64
+        const int zwords = PW * 32 * g.kw, xwords = TC_BM * g.kw;   // factor words of a panel / of the 128 rows
+        // 16-byte copies need 16-byte aligned sources: tile bases are, unless a tile holds an odd word count
+        const bool z_vec = ((g.tn * g.kw) & 3) == 0, x_vec = ((g.tm * g.kw) & 3) == 0;
 
-        struct PanelAt { const uint32_t *iz_tile; const uint32_t *ip_row; int c0; int j0; bool live; };
-        auto panel_at = [&](int P) {
-            PanelAt p;
-            p.live = P < npanels;
-            p.c0 = (kb_begin + P * KBP) * TC_BK;        // first column of the panel
-            const int tc = p.live ? p.c0 / g.tn : 0;
-            p.j0 = p.c0 - tc * g.tn;                    // ... inside its tile
+        // Stage the factor words of panel P: Iz words of its PW*32 columns, Ip words of the 128 rows.
+        // Words outside the tile are written as zero.  Asynchronous copies; the caller waits for them.
+        auto stage_factors = [&](int P) {
+            if (P >= npanels) return;
+            if (o0 >= g.rows) {                          // a block without rows of W (second CTA of a ragged pair)
+                for (int q = dt; q < zwords; q += TC_DECODE_WARPS * 32) iz_stage[q] = 0u;
+                for (int q = dt; q < xwords; q += TC_DECODE_WARPS * 32) ip_stage[q] = 0u;
+                return;
+            }
+            const int c0 = (kb_begin + P * KBP) * TC_BK;            // first column of the panel
+            const int tc = c0 / g.tn, j0 = c0 - tc * g.tn;           // ... its tile column, column inside the tile
             const size_t tile = (size_t)tr * g.gc + tc;
-            p.iz_tile = iz + tile * g.tn * g.kw;
-            p.ip_row = ip + (tile * g.tm + (row_ok ? i_row : 0)) * g.kw;
-            return p;
+            const uint32_t *zsrc = iz + (tile * g.tn + j0) * g.kw;
+            const uint32_t *xsrc = ip + (tile * g.tm + i0) * g.kw;
+            const int zvalid = (g.tn - j0) * g.kw, xvalid = (g.tm - i0) * g.kw;   // words that exist in the tile
+            for (int q = dt * 4; q < zwords; q += TC_DECODE_WARPS * 32 * 4) {
+                const int n = min(4, max(0, zvalid - q));
+                if (z_vec) cp_async_16(iz_stage + q, zsrc + (n > 0 ? q : 0), n * 4);
+                else for (int e = 0; e < 4; ++e) iz_stage[q + e] = e < n ? __ldg(zsrc + q + e) : 0u;
+            }
+            for (int q = dt * 4; q < xwords; q += TC_DECODE_WARPS * 32 * 4) {
+                const int n = min(4, max(0, xvalid - q));
+                if (x_vec) cp_async_16(ip_stage + q, xsrc + (n > 0 ? q : 0), n * 4);
+                else for (int e = 0; e < 4; ++e) ip_stage[q + e] = e < n ? __ldg(xsrc + q + e) : 0u;
+            }
+            cp_async_commit();
         };
-        auto load_z = [&](const PanelAt &p, int n) -> uint32_t {     // column word of pair dw + 4n, this lane's column
-            const int pi = dw + TC_DECODE_WARPS * n;
-            if (!p.live || pi >= npairs) return 0u;
-            const int lb = pi / PW, off = (pi % PW) * 32 + bit_col;
-            uint32_t z = 0;
-            if (p.c0 + off < g.cols && p.j0 + off < g.tn) z = __ldg(p.iz_tile + (p.j0 + off) * g.kw + lb);
-            return (lb == g.kw - 1) ? (z & tail) : z;
-        };
-        auto load_ip = [&](const PanelAt &p, int lb) -> uint32_t {   // row word lb of this thread's row
-            if (!p.live || !row_ok || lb >= g.kw) return 0u;
-            const uint32_t x = __ldg(p.ip_row + lb);
-            return (lb == g.kw - 1) ? (x & tail) : x;
-        };
-        // statically indexed only (fully unrolled loops): they stay in registers while loads are in flight
-        uint32_t zreg[ZREG], xreg[XREG];
-        {
-            const PanelAt p0 = panel_at(0);
-#pragma unroll
-            for (int n = 0; n < ZREG; ++n) zreg[n] = pre ? load_z(p0, n) : 0u;
-#pragma unroll
-            for (int lb = 0; lb < XREG; ++lb) xreg[lb] = pre ? load_ip(p0, lb) : 0u;
-        }
+
         uint32_t dsync_parity = 0;
         bool ok = true;
-        for (int P = 0; P < npanels && ok; ++P) {
-            const int buf = P & 1;
-            uint32_t *pl_buf = planes + buf * (g.kw * 32 * PW);
-            uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
-            // the pruning warps must be done with the panel that used this buffer two panels ago
-            ok = mbar_wait(&ctl->bits_free[buf], ((P >> 1) & 1) ^ 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
-            if (!ok) break;
-            // (a) bit-planes of Iz: each lane brings the k-bit word of one column, a warp-wide
-            //     transpose turns 32 column words into 32 plane words (lane l keeps plane lb*32 + l)
-            const PanelAt pc = panel_at(P), pn = panel_at(P + 1);
-            uint32_t xcur[XREG];
-            if (pre) {
-#pragma unroll
-                for (int n = 0; n < ZREG; ++n) {
-                    const int pi = dw + TC_DECODE_WARPS * n;
-                    if (pi < npairs) pl_buf[((pi / PW) * 32 + lane) * PW + (pi % PW)] = transpose32(zreg[n], lane);
-                }
-#pragma unroll
-                for (int lb = 0; lb < XREG; ++lb) xcur[lb] = xreg[lb];
-                // next panel's factor words start their trip now
-#pragma unroll
-                for (int n = 0; n < ZREG; ++n) zreg[n] = load_z(pn, n);
-#pragma unroll
-                for (int lb = 0; lb < XREG; ++lb) xreg[lb] = load_ip(pn, lb);
-            } else {
-                for (int n = 0; dw + TC_DECODE_WARPS * n < npairs; ++n) {
-                    const int pi = dw + TC_DECODE_WARPS * n;
-                    pl_buf[((pi / PW) * 32 + lane) * PW + (pi % PW)] = transpose32(load_z(pc, n), lane);
-                }
-            }
+        auto dsync = [&]() {                            // the four decoder warps meet (bounded wait)
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->dsync);
             ok = mbar_wait(&ctl->dsync, dsync_parity, abort_flag, status, DEV_TIMEOUT_EMPTY);
             dsync_parity ^= 1;
+        };
+
+        stage_factors(0);
+        for (int P = 0; P < npanels && ok; ++P) {
+            const int buf = P & 1;
+            uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
+            const int c0 = (kb_begin + P * KBP) * TC_BK;
+            cp_async_wait_all();                         // this thread's copies for panel P have landed
+            dsync();                                     // ... and everybody else's
+            if (!ok) break;
+            // (a) bit-planes of Iz: each lane brings the k-bit word of one column, a warp-wide transpose
+            //     turns 32 column words into 32 plane words (lane l keeps plane lb*32 + l)
+            for (int n0 = 0; dw + TC_DECODE_WARPS * n0 < npairs; n0 += 4) {
+                uint32_t z[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int pi = dw + TC_DECODE_WARPS * (n0 + t);
+                    const int lb = pi / PW, col = (pi % PW) * 32 + bit_col;
+                    z[t] = (pi < npairs && c0 + col < g.cols) ? iz_stage[col * g.kw + lb] : 0u;
+                    if (lb == g.kw - 1) z[t] &= tail;
+                }
+                transpose32_x4(z, lane);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int pi = dw + TC_DECODE_WARPS * (n0 + t);
+                    if (pi < npairs) planes[((pi / PW) * 32 + lane) * PWS + (pi % PW)] = z[t];
+                }
+            }
+            // this thread's row words of Ip, into registers (k <= 256: at most eight)
+            uint32_t xw[8];
+#pragma unroll
+            for (int lb = 0; lb < 8; ++lb) {
+                xw[lb] = (row_ok && lb < g.kw) ? ip_stage[dt * g.kw + lb] : 0u;
+                if (lb == g.kw - 1) xw[lb] &= tail;
+            }
+            dsync();                                     // planes complete, factor staging consumed
+            if (!ok) break;
+            stage_factors(P + 1);                        // next panel's factor words start their trip now
+            // the pruning warps must be done with the panel that used this buffer two panels ago
+            ok = mbar_wait(&ctl->bits_free[buf], ((P >> 1) & 1) ^ 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
             if (!ok) break;
             // (b) Eq. 3 for one row: OR of the planes its Ip bits select
             uint32_t acc[PW];
 #pragma unroll
             for (int q = 0; q < PW; ++q) acc[q] = 0;
-            auto or_planes = [&](uint32_t x, int lb) {
+#pragma unroll
+            for (int lb = 0; lb < 8; ++lb) {
+                uint32_t x = xw[lb];
                 while (x) {
                     const int l = lb * 32 + __ffs(x) - 1;
                     x &= x - 1;
-                    const uint32_t *src = pl_buf + l * PW;
+                    const uint32_t *src = planes + l * PWS;
                     if (PW == 8) {
                         const uint4 v0 = reinterpret_cast<const uint4 *>(src)[0], v1 = reinterpret_cast<const uint4 *>(src)[1];
                         acc[0] |= v0.x; acc[1] |= v0.y; acc[2 % PW] |= v0.z; acc[3 % PW] |= v0.w;
@@ -427,12 +545,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                         for (int q = 0; q < PW; ++q) acc[q] |= src[q];
                     }
                 }
-            };
-            if (pre) {
-#pragma unroll
-                for (int lb = 0; lb < XREG; ++lb) or_planes(xcur[lb], lb);
-            } else {
-                for (int lb = 0; lb < g.kw; ++lb) or_planes(load_ip(pc, lb), lb);
             }
             if (PW == 8) {
                 reinterpret_cast<uint4 *>(rb_buf + dt * PW)[0] = make_uint4(acc[0], acc[1], acc[2 % PW], acc[3 % PW]);
@@ -444,6 +556,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->bits_ready[buf]);
         }
+        cp_async_wait_all();
     } else {
         // ------------------------------------------------------------- pruning warps
         const int mt = threadIdx.x - 64;                // 0..255
@@ -502,50 +615,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         if (ok) {
             tc_fence_after();
             // All MMAs have completed, so the operand stages are free: reuse them to transpose the
-            // accumulator (lane = output feature) into rows of Y (contiguous output features).
+            // accumulator (lane = output feature) into rows of Y (contiguous output features).  The
+            // accumulator goes through in passes of at most 64 batch columns (128 x 64 x 4 bytes = 32 KB,
+            // which every stage configuration has room for).
             const bool out32 = partials != nullptr || y_dtype == LRBI_Y_F32;
+            const int esz = out32 ? 4 : 2;
             const int quad = warp & 3;                   // tensor-memory lanes this warp may read
-            const int half = mw >> 2;                    // which half of the accumulator columns
+            const int half = mw >> 2;                    // which half of a pass's columns
             const int ol = quad * 32 + lane;             // output feature inside the block
-            constexpr int COLS_PER_WARP = BN / 2 < 16 ? 16 : BN / 2;
+            constexpr int PASS = BN < 64 ? BN : 64;      // batch columns per pass
+            constexpr int COLS_PER_WARP = PASS / 2 < 16 ? 16 : PASS / 2;
             constexpr int NCHUNK = COLS_PER_WARP / 16;
-            if ((BN >= 32) || half == 0) {
+            uint8_t *dst_base = partials ? reinterpret_cast<uint8_t *>(partials + (long long)blockIdx.z * batch * g.rows)
+                                         : reinterpret_cast<uint8_t *>(Y);
+            const int row_bytes = TC_BM * esz;           // one batch row of the block
+            const int chunks = row_bytes / 16;           // 16 (bf16) or 32 (fp32)
+            const int per16 = 16 / esz;                  // outputs per 16-byte chunk
+            const bool vec_ok = (g.rows % per16) == 0;   // rows of Y stay 16-byte aligned
+            auto meet = [&]() {                          // the eight warps meet (bounded wait)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->epi);
+                ok = mbar_wait(&ctl->epi, epi_parity, abort_flag, status, DEV_TIMEOUT_ACCUM);
+                epi_parity ^= 1;
+            };
 #pragma unroll 1
-                for (int ch = 0; ch < NCHUNK; ++ch) {
-                    const int col0 = half * COLS_PER_WARP + ch * 16;
-                    uint32_t v[16];
-                    tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)col0, v);
-                    tmem_ld_wait();
-                    if (out32) {
-                        float *st = reinterpret_cast<float *>(smem);
+            for (int pass0 = 0; pass0 < BN && ok; pass0 += PASS) {
+                if ((PASS >= 32) || half == 0) {
+#pragma unroll 1
+                    for (int ch = 0; ch < NCHUNK; ++ch) {
+                        const int cl = half * COLS_PER_WARP + ch * 16;       // column inside the pass
+                        uint32_t v[16];
+                        tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass0 + cl), v);
+                        tmem_ld_wait();
+                        if (out32) {
+                            float *st = reinterpret_cast<float *>(smem);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) st[(col0 + j) * TC_BM + ol] = __uint_as_float(v[j]);
-                    } else {
-                        uint16_t *st = reinterpret_cast<uint16_t *>(smem);
+                            for (int j = 0; j < 16; ++j) st[(cl + j) * TC_BM + ol] = __uint_as_float(v[j]);
+                        } else {
+                            uint16_t *st = reinterpret_cast<uint16_t *>(smem);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) st[(col0 + j) * TC_BM + ol] = f32_to_bf16_rne(__uint_as_float(v[j]));
+                            for (int j = 0; j < 16; ++j) st[(cl + j) * TC_BM + ol] = f32_to_bf16_rne(__uint_as_float(v[j]));
+                        }
                     }
                 }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->epi);
-            ok = mbar_wait(&ctl->epi, epi_parity, abort_flag, status, DEV_TIMEOUT_ACCUM);
-            epi_parity ^= 1;
-            if (ok) {
-                const int esz = out32 ? 4 : 2;
-                uint8_t *dst_base = partials ? reinterpret_cast<uint8_t *>(partials + (long long)blockIdx.z * batch * g.rows)
-                                             : reinterpret_cast<uint8_t *>(Y);
-                const int row_bytes = TC_BM * esz;                       // one batch row of the block
-                const int chunks = row_bytes / 16;                       // 16 (bf16) or 32 (fp32)
-                const int per16 = 16 / esz;                              // outputs per 16-byte chunk
-                const int nb = min(BN, batch - b0);
-                const bool vec_ok = (g.rows % per16) == 0;               // rows of Y stay 16-byte aligned
+                meet();                                  // the pass is staged
+                if (!ok) break;
+                const int nb = min(PASS, batch - b0 - pass0);
                 for (int idx = mt; idx < nb * chunks; idx += TC_MASK_WARPS * 32) {
                     const int bl = idx / chunks, cj = idx - bl * chunks;
-                    const int oc = o0 + cj * per16;                      // first output feature of the chunk
+                    const int oc = o0 + cj * per16;      // first output feature of the chunk
                     if (oc >= g.rows) continue;
                     const uint8_t *src = smem + (size_t)bl * row_bytes + cj * 16;
-                    uint8_t *dst = dst_base + ((long long)(b0 + bl) * g.rows + oc) * esz;
+                    uint8_t *dst = dst_base + ((long long)(b0 + pass0 + bl) * g.rows + oc) * esz;
                     if (vec_ok && oc + per16 <= g.rows) {
                         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
                     } else {
@@ -554,15 +675,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                             *reinterpret_cast<uint16_t *>(dst + e) = *reinterpret_cast<const uint16_t *>(src + e);
                     }
                 }
+                if (pass0 + PASS < BN) meet();           // staging may be overwritten by the next pass
             }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();    // neither CTA frees tensor memory or leaves while the other may still touch it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_d, TMEM_COLS);
+        if (PAIR) tmem_dealloc2(tmem_d, TMEM_COLS);
+        else tmem_dealloc(tmem_d, TMEM_COLS);
     }
 }
 
@@ -632,7 +756,7 @@ static float *workspace(size_t bytes)
     return w.ptr;
 }
 
-template <int BN, int PW>
+template <int BN, int PW, bool PAIR>
 static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                              const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count)
 {
@@ -641,7 +765,7 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.cols, (cuuint64_t)batch};
     const cuuint64_t strides[1] = {(cuuint64_t)g.cols * 2};
-    const cuuint32_t box[2] = {TC_BK, BN};
+    const cuuint32_t box[2] = {TC_BK, PAIR ? BN / 2 : BN};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -655,9 +779,10 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
-    constexpr int B_STAGE = BN * TC_BK * 2;
+    constexpr int B_STAGE = (PAIR ? BN / 2 : BN) * TC_BK * 2;
     const int nkb = (g.cols + TC_BK - 1) / TC_BK;
-    const int tiles = ((batch + BN - 1) / BN) * ((g.rows + TC_BM - 1) / TC_BM);
+    const int row_blocks = PAIR ? 2 * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) : (g.rows + TC_BM - 1) / TC_BM;
+    const int tiles = ((batch + BN - 1) / BN) * row_blocks;
     // split K when the output tiles alone cannot occupy the chip (small batch: bandwidth-bound)
     int splits = 1;
     if (batch <= BN && tiles < 2 * sm_count) {        // one batch tile: the small-batch, bandwidth-bound case
@@ -669,28 +794,45 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     kb_per_split = (kb_per_split + 3) / 4 * 4;                               // splits start on panel boundaries
     splits = (nkb + kb_per_split - 1) / kb_per_split;                        // no empty split
 
-    int stages = BN >= 256 ? 4 : (BN >= 128 ? 4 : 6);
-    if (stages > 8) stages = 8;
-    const size_t smem = 1024 + (size_t)stages * (TC_A_STAGE_BYTES + B_STAGE) + (size_t)2 * (TC_BM + g.kw * 32) * PW * 4 + sizeof(TcCtl);
+    // Pair mode: three stages when two blocks then fit one SM (k <= 64); larger ranks need more room for
+    // planes and factor staging, run one block per SM and get six stages.
+    const size_t extras = (size_t)(2 * TC_BM * PW + g.kw * 32 * (PW == 8 ? 12 : PW) + PW * 32 * g.kw + TC_BM * g.kw) * 4 + sizeof(TcCtl);
+    const size_t per_stage = TC_A_STAGE_BYTES + B_STAGE;
+    int stages = BN >= 128 ? 4 : 6;
+    if (PAIR) stages = (3 * per_stage + extras <= 114 * 1024) ? 3 : 6;
+    const size_t smem = (size_t)stages * per_stage + extras;
 
     float *partials = nullptr;
     if (splits > 1) {
         partials = workspace((size_t)splits * batch * g.rows * sizeof(float));
         if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
     }
-    auto kern = gemm_tc_kernel<BN, PW>;
+    auto kern = gemm_tc_kernel<BN, PW, PAIR>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
         attr_done = true;
     }
-    dim3 grid((unsigned)((batch + BN - 1) / BN), (unsigned)((g.rows + TC_BM - 1) / TC_BM), (unsigned)splits);
+    const unsigned nbt = (unsigned)((batch + BN - 1) / BN);
+    dim3 grid(PAIR ? 2 * nbt : nbt, (unsigned)(PAIR ? row_blocks / 2 : row_blocks), (unsigned)splits);
     if (grid.y > 65535 || grid.z > 65535) return LRBI_ERR_UNSUPPORTED;
-    kern<<<grid, TC_THREADS, smem, s>>>(map, wmap, g, ip, iz, batch, Y, y_dtype, partials, kb_per_split, stages,
-                                         device_status_ptr());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;      // the pair must lie along x: other shapes are refused
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int *status = device_status_ptr();
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, ip, iz, batch, Y, y_dtype, partials, kb_per_split, stages, status);
     count_launch();
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
     if (splits > 1) {
         const long long n = (long long)batch * g.rows;
@@ -706,8 +848,8 @@ template <int BN>
 static lrbi_status launch_tc_kw(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                                 const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count)
 {
-    return panel_words(g) == 8 ? launch_tc<BN, 8>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
-                               : launch_tc<BN, 2>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    return panel_words(g) == 8 ? launch_tc<BN, 8, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
+                               : launch_tc<BN, 2, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
 }
 
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
@@ -722,7 +864,9 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
     if (batch <= 32) return launch_tc_kw<32>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
     if (batch <= 64) return launch_tc_kw<64>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
     if (batch <= 128) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    return launch_tc_kw<256>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    // large batch: CTA pairs share each X tile
+    return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
+                               : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
 }
 
 }  // namespace lrbi
