@@ -52,7 +52,8 @@ typedef enum {
     LRBI_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer          */
     LRBI_ERR_UNSUPPORTED = 2, /* a shape, dtype or kernel choice this build does not cover     */
     LRBI_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed (see lrbi_last_cuda_error)  */
-    LRBI_ERR_TIMEOUT = 4      /* a bounded device-side wait gave up (see lrbi_device_status)   */
+    LRBI_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up (see lrbi_device_status)   */
+    LRBI_ERR_TOO_LARGE = 5    /* the problem needs more fixed scratch than the library carries   */
 } lrbi_status;
 
 /* Geometry of one pruned layer (Section 3.1: equal tiles, one rank). */
@@ -112,6 +113,39 @@ LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t 
 LRBI_API lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const uint32_t *ip,
                              const uint32_t *iz, const uint16_t *X, int32_t batch, void *Y,
                              int32_t y_dtype, int32_t algo, void *stream);
+
+/*
+ * lrbi_masked_gemm for callers that must not allocate device memory.  (The paper has no
+ * counterpart to this call; it exists for the library's users.)
+ *
+ * Who needs it: code that runs inside a memory-pool or arena discipline where every device byte
+ * is accounted for up front (an inference server that sizes its pool at start-up and treats a
+ * later cudaMalloc as a bug), code that runs where cudaMalloc may block or fail at a bad moment
+ * (it takes a device-wide lock and can synchronise; under memory pressure it returns an error in
+ * the middle of a request), and plug-ins that are simply not given the right to allocate.
+ * lrbi_masked_gemm may allocate: when it splits the reduction over K it keeps fp32 partial sums
+ * in a buffer that it grows with cudaMalloc.  This call never does.  It always runs the
+ * tensor-core kernel (LRBI_ALGO_TENSOR shapes only, else LRBI_ERR_UNSUPPORTED) and keeps the
+ * partial sums in a fixed array that is part of the library image: LRBI_STATIC_SCRATCH_BYTES
+ * (8 MiB) of device memory on every GPU that loads the library, held until the process exits.
+ *
+ *   - If splits * batch * rows * 4 bytes exceeds that array the call returns LRBI_ERR_TOO_LARGE
+ *     and launches nothing (lrbi_masked_gemm_static_bytes tells the need in advance; 0 = no
+ *     scratch needed).  Large batches do not split K and need none.
+ *   - It calls no cudaMalloc, cudaFree or any other allocating routine.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current) and caches it; make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left in it.
+ *     Nothing has to be cleared: every word the reduction reads was written earlier in the same
+ *     call.  But two calls that overlap on the GPU (different streams) race on it and give wrong
+ *     results: keep calls to this entry point on one stream, or order them with events.
+ * Arguments, layouts and results are those of lrbi_masked_gemm with LRBI_ALGO_TENSOR.
+ */
+#define LRBI_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+LRBI_API lrbi_status lrbi_masked_gemm_static(const lrbi_layout *layout, const uint16_t *W, const uint32_t *ip,
+                                             const uint32_t *iz, const uint16_t *X, int32_t batch, void *Y,
+                                             int32_t y_dtype, void *stream);
+LRBI_API size_t lrbi_masked_gemm_static_bytes(const lrbi_layout *layout, int32_t batch);
 
 /*
  * Same computation for callers whose activations live in host memory (the index and the

@@ -21,7 +21,8 @@ LIB_PATH = os.path.join(_HERE, "liblrbi.so")
 ALGO_AUTO, ALGO_GENERIC, ALGO_GEMV, ALGO_TENSOR, ALGO_DECODE_BALLOT, ALGO_DECODE_PLANES = range(6)
 ALGO_NAMES = {0: "auto", 1: "generic", 2: "gemv", 3: "tensor", 4: "decode_ballot", 5: "decode_planes"}
 Y_BF16, Y_F32 = 0, 1
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = range(5)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(6)
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
 class LrbiError(RuntimeError):
@@ -62,6 +63,10 @@ def lib():
         L.lrbi_decode_mask.restype = i32
         L.lrbi_masked_gemm.argtypes = [lp, vp, vp, vp, vp, i32, vp, i32, i32, vp]
         L.lrbi_masked_gemm.restype = i32
+        L.lrbi_masked_gemm_static.argtypes = [lp, vp, vp, vp, vp, i32, vp, i32, vp]
+        L.lrbi_masked_gemm_static.restype = i32
+        L.lrbi_masked_gemm_static_bytes.argtypes = [lp, i32]
+        L.lrbi_masked_gemm_static_bytes.restype = ctypes.c_size_t
         L.lrbi_layer_create.argtypes = [lp, vp, vp, vp, i32, ctypes.POINTER(vp)]
         L.lrbi_layer_create.restype = i32
         L.lrbi_layer_forward_host.argtypes = [vp, vp, i32, vp, i32, i32]
@@ -159,6 +164,36 @@ def lrbi_masked_gemm(layer, W: torch.Tensor, ip: torch.Tensor, iz: torch.Tensor,
                             _dev(Y, Y.dtype, "Y"), code, algo, _stream_ptr(stream))
     if rc != OK:
         raise LrbiError(rc, "lrbi_masked_gemm")
+    return Y
+
+
+def masked_gemm_static_bytes(layer, batch: int) -> int:
+    """Bytes of the fixed scratch array lrbi_masked_gemm_static would use for this call (0 = none)."""
+    lay = Layout.of(layer)
+    return int(lib().lrbi_masked_gemm_static_bytes(ctypes.byref(lay), batch))
+
+
+def lrbi_masked_gemm_static(layer, W: torch.Tensor, ip: torch.Tensor, iz: torch.Tensor, X: torch.Tensor,
+                            Y: torch.Tensor, stream=None) -> torch.Tensor:
+    """lrbi_masked_gemm for callers that may not allocate device memory.
+
+    The library call allocates nothing: its K-split partial sums go to a fixed 8 MiB array inside the
+    library.  That is why Y is not optional here: a caller that cannot allocate brings its output.
+    Raises LrbiError with code ERR_TOO_LARGE if the fixed array is too small.  Calls share that array:
+    keep them on one stream.
+    """
+    lay = Layout.of(layer)
+    batch = X.shape[0]
+    if tuple(W.shape) != (lay.rows, lay.cols) or X.dim() != 2 or X.shape[1] != lay.cols:
+        raise ValueError("W / X shapes do not match the layout")
+    if tuple(Y.shape) != (batch, lay.rows) or Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y must be [batch, rows] bf16 or fp32")
+    code = Y_BF16 if Y.dtype == torch.bfloat16 else Y_F32
+    rc = lib().lrbi_masked_gemm_static(ctypes.byref(lay), _dev(W, torch.bfloat16, "W"), _dev(ip, torch.int32, "ip"),
+                                       _dev(iz, torch.int32, "iz"), _dev(X, torch.bfloat16, "X"), batch,
+                                       _dev(Y, Y.dtype, "Y"), code, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_masked_gemm_static")
     return Y
 
 

@@ -113,6 +113,23 @@ lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const
     }
 }
 
+lrbi_status lrbi_masked_gemm_static(const lrbi_layout *layout, const uint16_t *W, const uint32_t *ip,
+                                    const uint32_t *iz, const uint16_t *X, int32_t batch, void *Y,
+                                    int32_t y_dtype, void *stream)
+{
+    if (!layout_ok(layout) || !W || !ip || !iz || !X || !Y || batch < 1) return LRBI_ERR_INVALID_ARG;
+    if (y_dtype != LRBI_Y_BF16 && y_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(ip) || !aligned16(iz) || !aligned16(X) || !aligned16(Y)) return LRBI_ERR_INVALID_ARG;
+    return launch_gemm_tc_static(make_geo(*layout), W, ip, iz, X, batch, Y, y_dtype, static_cast<cudaStream_t>(stream));
+}
+
+size_t lrbi_masked_gemm_static_bytes(const lrbi_layout *layout, int32_t batch)
+{
+    if (!layout_ok(layout) || batch < 1) return 0;
+    const Geo g = make_geo(*layout);
+    return gemm_tc_supported(g, batch) ? gemm_tc_scratch_bytes(g, batch) : 0;
+}
+
 uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t lrbi_device_status(int32_t clear)
@@ -138,6 +155,7 @@ const char *lrbi_status_string(lrbi_status s)
     case LRBI_ERR_UNSUPPORTED: return "unsupported shape or kernel choice";
     case LRBI_ERR_CUDA: return "CUDA call failed";
     case LRBI_ERR_TIMEOUT: return "device-side wait timed out";
+    case LRBI_ERR_TOO_LARGE: return "needs more scratch than the fixed array holds";
     default: return "unknown status";
     }
 }

@@ -756,9 +756,32 @@ static float *workspace(size_t bytes)
     return w.ptr;
 }
 
+// How the reduction over K is cut: `splits` blocks along grid z, each `kb_per_split` K blocks long.
+struct SplitPlan { int splits, kb_per_split, row_blocks; };
+static SplitPlan plan_splits(const Geo &g, int batch, int bn, bool pair, int sm_count)
+{
+    SplitPlan p;
+    const int nkb = (g.cols + TC_BK - 1) / TC_BK;
+    p.row_blocks = pair ? 2 * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) : (g.rows + TC_BM - 1) / TC_BM;
+    const int tiles = ((batch + bn - 1) / bn) * p.row_blocks;
+    // split K when the output tiles alone cannot occupy the chip (small batch: bandwidth-bound)
+    int splits = 1;
+    if (batch <= bn && tiles < 2 * sm_count) {        // one batch tile: the small-batch, bandwidth-bound case
+        splits = (2 * sm_count + tiles - 1) / tiles;
+        splits = splits > nkb / 4 ? (nkb / 4 > 0 ? nkb / 4 : 1) : splits;   // at least 4 K blocks per split
+        if (splits > 32) splits = 32;
+    }
+    int kb_per_split = (nkb + splits - 1) / splits;
+    kb_per_split = (kb_per_split + 3) / 4 * 4;                               // splits start on panel boundaries
+    p.splits = (nkb + kb_per_split - 1) / kb_per_split;                      // no empty split
+    p.kb_per_split = kb_per_split;
+    return p;
+}
+
 template <int BN, int PW, bool PAIR>
 static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                             const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count)
+                             const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count,
+                             float *fixed_scratch = nullptr, size_t fixed_bytes = 0)
 {
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) { note_cuda_error(-1); return LRBI_ERR_CUDA; }
@@ -780,19 +803,8 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
     constexpr int B_STAGE = (PAIR ? BN / 2 : BN) * TC_BK * 2;
-    const int nkb = (g.cols + TC_BK - 1) / TC_BK;
-    const int row_blocks = PAIR ? 2 * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) : (g.rows + TC_BM - 1) / TC_BM;
-    const int tiles = ((batch + BN - 1) / BN) * row_blocks;
-    // split K when the output tiles alone cannot occupy the chip (small batch: bandwidth-bound)
-    int splits = 1;
-    if (batch <= BN && tiles < 2 * sm_count) {        // one batch tile: the small-batch, bandwidth-bound case
-        splits = (2 * sm_count + tiles - 1) / tiles;
-        splits = splits > nkb / 4 ? (nkb / 4 > 0 ? nkb / 4 : 1) : splits;   // at least 4 K blocks per split
-        if (splits > 32) splits = 32;
-    }
-    int kb_per_split = (nkb + splits - 1) / splits;
-    kb_per_split = (kb_per_split + 3) / 4 * 4;                               // splits start on panel boundaries
-    splits = (nkb + kb_per_split - 1) / kb_per_split;                        // no empty split
+    const SplitPlan plan = plan_splits(g, batch, BN, PAIR, sm_count);
+    const int row_blocks = plan.row_blocks, splits = plan.splits, kb_per_split = plan.kb_per_split;
 
     // Pair mode: three stages when two blocks then fit one SM (k <= 64); larger ranks need more room for
     // planes and factor staging, run one block per SM and get six stages.
@@ -804,8 +816,14 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
 
     float *partials = nullptr;
     if (splits > 1) {
-        partials = workspace((size_t)splits * batch * g.rows * sizeof(float));
-        if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
+        const size_t need = (size_t)splits * batch * g.rows * sizeof(float);
+        if (fixed_scratch) {                             // caller forbids allocation: fixed array or nothing
+            if (need > fixed_bytes) return LRBI_ERR_TOO_LARGE;
+            partials = fixed_scratch;
+        } else {
+            partials = workspace(need);
+            if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
+        }
     }
     auto kern = gemm_tc_kernel<BN, PW, PAIR>;
     static bool attr_done = false;
@@ -846,10 +864,11 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
 
 template <int BN>
 static lrbi_status launch_tc_kw(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                                const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count)
+                                const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count,
+                                float *fixed_scratch = nullptr, size_t fixed_bytes = 0)
 {
-    return panel_words(g) == 8 ? launch_tc<BN, 8, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
-                               : launch_tc<BN, 2, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    return panel_words(g) == 8 ? launch_tc<BN, 8, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, fixed_scratch, fixed_bytes)
+                               : launch_tc<BN, 2, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, fixed_scratch, fixed_bytes);
 }
 
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
@@ -867,6 +886,59 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
     // large batch: CTA pairs share each X tile
     return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
                                : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+}
+
+// --------------------------------------------------------------------------------------
+// No-allocation variant: K-split partial sums live in a fixed array inside the library image.
+// --------------------------------------------------------------------------------------
+// The array belongs to the module: each GPU that loads the library carries its own copy until the
+// process ends.  In host code this name is only a handle for the runtime, never a device address;
+// the address a kernel may use comes from cudaGetSymbolAddress, asked once per device.
+static __device__ __align__(256) float g_static_scratch[LRBI_STATIC_SCRATCH_BYTES / sizeof(float)];
+static float *g_static_scratch_ptr[64] = {nullptr};
+
+static float *static_scratch_ptr()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!g_static_scratch_ptr[dev]) {                    // first call on this device (it is the current one)
+        void *p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) { note_cuda_error((int)e); return nullptr; }
+        g_static_scratch_ptr[dev] = static_cast<float *>(p);
+    }
+    return g_static_scratch_ptr[dev];
+}
+
+static int batch_tile(int batch) { return batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : batch <= 128 ? 128 : 256; }
+
+size_t gemm_tc_scratch_bytes(const Geo &g, int batch)
+{
+    int dev = 0, sm_count = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    const SplitPlan p = plan_splits(g, batch, batch_tile(batch), batch > 128, sm_count);
+    return p.splits > 1 ? (size_t)p.splits * batch * g.rows * sizeof(float) : 0;
+}
+
+lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                                  const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s)
+{
+    if (!gemm_tc_supported(g, batch)) return LRBI_ERR_UNSUPPORTED;
+    if (gemm_tc_scratch_bytes(g, batch) > LRBI_STATIC_SCRATCH_BYTES) return LRBI_ERR_TOO_LARGE;   // before any launch
+    if (!device_status_ptr()) return LRBI_ERR_CUDA;
+    float *scratch = static_scratch_ptr();
+    if (!scratch) return LRBI_ERR_CUDA;
+    int dev = 0, sm_count = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    const size_t cap = LRBI_STATIC_SCRATCH_BYTES;
+    if (batch <= 16) return launch_tc_kw<16>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
+    if (batch <= 32) return launch_tc_kw<32>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
+    if (batch <= 64) return launch_tc_kw<64>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
+    if (batch <= 128) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
+    return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap)
+                               : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
 }
 
 }  // namespace lrbi

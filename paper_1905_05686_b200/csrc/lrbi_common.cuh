@@ -74,4 +74,9 @@ bool gemm_tc_supported(const Geo &g, int batch);
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                            const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 
+// Variant that keeps K-split partial sums in the library's fixed device array; allocates nothing.
+lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                                  const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+size_t gemm_tc_scratch_bytes(const Geo &g, int batch);   // fp32 partial sums the tensor-core path would keep
+
 }  // namespace lrbi
