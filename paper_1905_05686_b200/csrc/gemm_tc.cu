@@ -308,7 +308,7 @@ __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
 // one tensor core pass instead of two.  Two such blocks are resident per SM (three stages each), so
 // one block's epilogue and panel hand-overs overlap the other's MMAs.
 template <int BN, int PW, bool PAIR>
-__global__ void __launch_bounds__(TC_THREADS, PAIR ? 2 : 1)
+__global__ void __launch_bounds__(TC_THREADS, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
@@ -810,8 +810,14 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     // planes and factor staging, run one block per SM and get six stages.
     const size_t extras = (size_t)(2 * TC_BM * PW + g.kw * 32 * (PW == 8 ? 12 : PW) + PW * 32 * g.kw + TC_BM * g.kw) * 4 + sizeof(TcCtl);
     const size_t per_stage = TC_A_STAGE_BYTES + B_STAGE;
-    int stages = BN >= 128 ? 4 : 6;
-    if (PAIR) stages = (3 * per_stage + extras <= 114 * 1024) ? 3 : 6;
+    // As many stages as let two blocks share an SM (at least three); if two cannot fit, one block with
+    // up to six stages.  Two resident blocks overlap one's epilogue and hand-overs with the other's MMAs
+    // and double the copies in flight.
+    const size_t half_sm = 114 * 1024, whole_sm = 224 * 1024;
+    int stages = (int)((half_sm - extras) / per_stage);
+    if (extras > half_sm || stages < 3) stages = (int)((whole_sm - extras) / per_stage);
+    if (stages > 6) stages = 6;
+    if (stages < 2) return LRBI_ERR_UNSUPPORTED;
     const size_t smem = (size_t)stages * per_stage + extras;
 
     float *partials = nullptr;
@@ -828,7 +834,7 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     auto kern = gemm_tc_kernel<BN, PW, PAIR>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
         if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
         attr_done = true;
     }
@@ -871,6 +877,13 @@ static lrbi_status launch_tc_kw(const Geo &g, const uint16_t *W, const uint32_t 
                                : launch_tc<BN, 2, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, fixed_scratch, fixed_bytes);
 }
 
+static bool use_pairs(const Geo &g, int batch, int sm_count)
+{
+    if (batch <= 128) return false;
+    const long long pair_blocks = 2LL * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) * ((batch + 255) / 256);
+    return pair_blocks * 2 >= 3LL * sm_count;
+}
+
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                            const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s)
 {
@@ -883,9 +896,12 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
     if (batch <= 32) return launch_tc_kw<32>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
     if (batch <= 64) return launch_tc_kw<64>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
     if (batch <= 128) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    // large batch: CTA pairs share each X tile
-    return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
-                               : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    // large batch: CTA pairs share each X tile, unless there are too few pairs of tiles to fill the chip
+    // (a layer with few rows): then single CTAs with 128-row batch tiles give twice as many blocks
+    if (use_pairs(g, batch, sm_count))
+        return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
+                                   : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
 }
 
 // --------------------------------------------------------------------------------------
@@ -917,7 +933,8 @@ size_t gemm_tc_scratch_bytes(const Geo &g, int batch)
     int dev = 0, sm_count = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    const SplitPlan p = plan_splits(g, batch, batch_tile(batch), batch > 128, sm_count);
+    const bool pair = use_pairs(g, batch, sm_count);
+    const SplitPlan p = plan_splits(g, batch, (batch > 128 && !pair) ? 128 : batch_tile(batch), pair, sm_count);
     return p.splits > 1 ? (size_t)p.splits * batch * g.rows * sizeof(float) : 0;
 }
 
@@ -936,7 +953,7 @@ lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_
     if (batch <= 16) return launch_tc_kw<16>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
     if (batch <= 32) return launch_tc_kw<32>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
     if (batch <= 64) return launch_tc_kw<64>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
-    if (batch <= 128) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
+    if (batch <= 128 || !use_pairs(g, batch, sm_count)) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
     return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap)
                                : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
 }
