@@ -813,7 +813,8 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     // As many stages as let two blocks share an SM (at least three); if two cannot fit, one block with
     // up to six stages.  Two resident blocks overlap one's epilogue and hand-overs with the other's MMAs
     // and double the copies in flight.
-    const size_t half_sm = 114 * 1024, whole_sm = 224 * 1024;
+    // (an SM has 228 KB of shared memory; each resident block also reserves 1 KB)
+    const size_t half_sm = 113 * 1024, whole_sm = 224 * 1024;
     int stages = (int)((half_sm - extras) / per_stage);
     if (extras > half_sm || stages < 3) stages = (int)((whole_sm - extras) / per_stage);
     if (stages > 6) stages = 6;
