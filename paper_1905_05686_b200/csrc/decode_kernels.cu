@@ -4,10 +4,13 @@
 //   decode_ballot  any shape.  A lane owns one column word of Iz, the row word of Ip is
 //                  warp-uniform, the test is (ip & iz) != 0 and __ballot_sync builds one
 //                  32-bit mask word per vote.  ~3 warp instructions per output word.
-//   decode_planes  tile_cols % 32 == 0.  Iz of a 256-column block is first transposed into k
-//                  bit-planes (plane l = 256 bits of row l of Iz) with __ballot_sync; a thread
-//                  then owns one mask row and ORs the planes selected by the set bits of its
-//                  Ip word: 32 mask bits per bitwise instruction instead of one per lane.
+//   decode_planes  tile_cols % 32 == 0.  Iz of a block of columns is first transposed into k
+//                  bit-planes (plane l = the bits of row l of Iz); a thread then owns one mask row
+//                  and ORs the planes selected by the set bits of its Ip word: 32 mask bits per
+//                  bitwise instruction instead of one per lane.  Two variants: 256-column blocks
+//                  transposed with __ballot_sync (any tile_cols % 32 == 0), and, for
+//                  tile_cols % 128 == 0 and k <= 256, 1024-column blocks transposed with warp
+//                  shuffles, where a thread writes whole 128-byte lines of its mask row.
 #include "lrbi_common.cuh"
 
 namespace lrbi {
@@ -189,10 +192,148 @@ decode_planes_kernel(Geo g, int col_blocks_per_tile, int row_bands_per_tile,
     }
 }
 
+// --------------------------------------------------------------------------------------
+// decode_planes, wide variant: a block decodes up to 1024 rows x 1024 columns
+// --------------------------------------------------------------------------------------
+constexpr int WIDE_WORDS = 32;          // mask words (1024 columns = one 128-byte line) per row and block
+constexpr int WIDE_PITCH = 36;          // words between planes in shared memory (16-byte aligned, spreads banks)
+constexpr int WIDE_MAX_RANK = 256;
+
+// 32 x 32 bit-matrix transpose across a warp: lane L gives x_L, lane l receives the word whose bit L is
+// bit l of x_L -- the 32 words that 32 __ballot_sync votes on ((x >> l) & 1) would give.
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane)
+{
+#pragma unroll
+    for (int stage = 0; stage < 5; ++stage) {
+        const int j = 16 >> stage;
+        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
+                         : stage == 3 ? 0x33333333u : 0x55555555u;
+        const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, j);
+        const bool upper = (lane & j) != 0;
+        const uint32_t sh = upper ? (y >> j) : (y << j);
+        const uint32_t keep = upper ? ~m : m;
+        x = (x & keep) | (sh & ~keep);
+    }
+    return x;
+}
+
+// SEGQ = 128-column quads per run of columns that lies inside one tile (8: the whole block).
+template <int SEGQ>
+__global__ void __launch_bounds__(DEC_THREADS)
+decode_planes_wide_kernel(Geo g, int row_bands_per_tile, int rows_per_block,
+                          const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz,
+                          uint32_t *__restrict__ mask)
+{
+    extern __shared__ __align__(16) uint32_t planes[];         // [kw*32][WIDE_PITCH]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gw0 = blockIdx.x * WIDE_WORDS;                    // first mask word of this block's columns
+    const int tr = blockIdx.y / row_bands_per_tile, band = blockIdx.y - tr * row_bands_per_tile;
+    const int words_in_tile = g.tn >> 5;
+    const uint32_t tail = tail_mask(g.k);
+    const int i_end = min(g.tm, g.rows - tr * g.tm);
+    const int i_first = band * rows_per_block + threadIdx.x;
+
+    // Row words of Ip for this thread's first row, requested before the planes are built so that their
+    // trip from memory overlaps the trip of the column words (k <= 64; larger ranks load them later).
+    constexpr int NSEG = 8 / SEGQ;
+    uint32_t xpre[NSEG][2];
+    const bool pre = g.kw <= 2;
+#pragma unroll
+    for (int seg = 0; seg < NSEG; ++seg) {
+        const int gw = gw0 + seg * SEGQ * 4;
+        const bool live = pre && gw < g.pitch && i_first < i_end;
+        const uint32_t *ipw = ip + (((long long)tr * g.gc + (live ? gw / words_in_tile : 0)) * g.tm + (live ? i_first : 0)) * g.kw;
+#pragma unroll
+        for (int lb = 0; lb < 2; ++lb) xpre[seg][lb] = (live && lb < g.kw) ? __ldg(ipw + lb) : 0u;
+    }
+
+    // ---- bit-planes of the block's 1024 columns: one warp transpose per (32 planes, mask word)
+    for (int pi = warp; pi < g.kw * WIDE_WORDS; pi += DEC_THREADS / 32) {
+        const int lb = pi / WIDE_WORDS, w = pi - lb * WIDE_WORDS;
+        const int c = (gw0 + w) * 32 + lane;                    // column of this lane
+        uint32_t z = 0;
+        if (c < g.cols) {
+            const int tc = c / g.tn, j = c - tc * g.tn;
+            z = __ldg(iz + (((long long)tr * g.gc + tc) * g.tn + j) * g.kw + lb);
+            if (lb == g.kw - 1) z &= tail;
+        }
+        planes[(lb * 32 + lane) * WIDE_PITCH + w] = warp_transpose32(z, lane);   // lane l keeps plane lb*32 + l
+    }
+    __syncthreads();
+
+    // ---- one thread per mask row; per run of quads inside one tile, OR the planes its Ip word selects
+    const bool vec = (g.pitch & 3) == 0;
+    for (int i = i_first; i < min(i_end, (band + 1) * rows_per_block); i += DEC_THREADS) {
+        uint4 acc[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc[q] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int seg = 0; seg < 8 / SEGQ; ++seg) {
+            const int gw = gw0 + seg * SEGQ * 4;                // first mask word of the run
+            if (gw >= g.pitch) break;
+            const int tc = gw / words_in_tile;
+            const uint32_t *ipw = ip + (((long long)tr * g.gc + tc) * g.tm + i) * g.kw;
+            auto or_planes = [&](uint32_t x, int lb) {
+                if (lb == g.kw - 1) x &= tail;
+                while (x) {
+                    const int l = lb * 32 + __ffs(x) - 1;
+                    x &= x - 1;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(planes + l * WIDE_PITCH + seg * SEGQ * 4);
+#pragma unroll
+                    for (int q = 0; q < SEGQ; ++q) {
+                        const uint4 v = src[q];
+                        uint4 &a = acc[seg * SEGQ + q];
+                        a.x |= v.x; a.y |= v.y; a.z |= v.z; a.w |= v.w;
+                    }
+                }
+            };
+            if (pre && i == i_first) {                   // statically indexed: the prefetched words stay in registers
+                or_planes(xpre[seg][0], 0);
+                if (g.kw > 1) or_planes(xpre[seg][1], 1);
+            } else {
+                for (int lb = 0; lb < g.kw; ++lb) or_planes(__ldg(ipw + lb), lb);
+            }
+        }
+        uint32_t *dst = mask + (long long)(tr * g.tm + i) * g.pitch + gw0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int nw = g.pitch - gw0 - q * 4;                // words of this quad that exist in the row
+            if (nw >= 4 && vec) {
+                reinterpret_cast<uint4 *>(dst)[q] = acc[q];
+            } else if (nw > 0) {
+                const uint32_t v[4] = {acc[q].x, acc[q].y, acc[q].z, acc[q].w};
+                for (int e = 0; e < min(nw, 4); ++e) dst[q * 4 + e] = v[e];
+            }
+        }
+    }
+}
+
+static bool decode_planes_wide_supported(const Geo &g) { return (g.tn % 128) == 0 && g.k <= WIDE_MAX_RANK; }
+
+static lrbi_status launch_decode_planes_wide(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask,
+                                             cudaStream_t s)
+{
+    const int rows_per_block = g.tm >= 1024 ? 1024 : (g.tm + DEC_THREADS - 1) / DEC_THREADS * DEC_THREADS;
+    const int rbpt = (g.tm + rows_per_block - 1) / rows_per_block;
+    dim3 grid((unsigned)((g.pitch + WIDE_WORDS - 1) / WIDE_WORDS), (unsigned)(g.gr * rbpt));
+    if (grid.y > 65535) return LRBI_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)g.kw * 32 * WIDE_PITCH * sizeof(uint32_t);       // <= 36 KB
+    const int segq = (g.tn % 1024) == 0 || g.gc == 1 ? 8 : (g.tn % 512) == 0 ? 4 : (g.tn % 256) == 0 ? 2 : 1;
+    if (segq == 8) decode_planes_wide_kernel<8><<<grid, DEC_THREADS, smem, s>>>(g, rbpt, rows_per_block, ip, iz, mask);
+    else if (segq == 4) decode_planes_wide_kernel<4><<<grid, DEC_THREADS, smem, s>>>(g, rbpt, rows_per_block, ip, iz, mask);
+    else if (segq == 2) decode_planes_wide_kernel<2><<<grid, DEC_THREADS, smem, s>>>(g, rbpt, rows_per_block, ip, iz, mask);
+    else decode_planes_wide_kernel<1><<<grid, DEC_THREADS, smem, s>>>(g, rbpt, rows_per_block, ip, iz, mask);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
+    return LRBI_OK;
+}
+
 lrbi_status launch_decode_planes(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask,
                                  cudaStream_t s)
 {
     if (!decode_planes_supported(g)) return LRBI_ERR_UNSUPPORTED;
+    if (decode_planes_wide_supported(g)) return launch_decode_planes_wide(g, ip, iz, mask, s);
     const int cbpt = ((g.tn >> 5) + DEC_WORDS - 1) / DEC_WORDS;
     const int rbpt = (g.tm + PLANES_ROWS_PER_BLOCK - 1) / PLANES_ROWS_PER_BLOCK;
     dim3 grid((unsigned)(g.gc * cbpt), (unsigned)(g.gr * rbpt));

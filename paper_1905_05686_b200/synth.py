@@ -66,6 +66,10 @@ CONFIGS = {
     "conv3x3_256": Layer("conv3x3_256", 256, 2304, 128, 256, 16, 0.30, 0.02, (12544,)),
     "ffn_16384x4096": Layer("ffn_16384x4096", 16384, 4096, 1024, 1024, 64, 0.20, 0.02, (4096,)),
 }
+# Not one of the five layer shapes: the decode-only configuration repeated over a grid 64 times larger
+# (same 256 x 256 tiles, rank and density; 128 MiB of mask), so that a decode kernel's steady-state
+# bandwidth can be measured on something larger than L2.
+CONFIGS["decode_32768"] = Layer("decode_32768", 32768, 32768, 256, 256, 8, 0.10, 0.0, ())
 CONFIG_ORDER = ["lenet_fc1", "decode_4096", "alexnet_fc", "conv3x3_256", "ffn_16384x4096"]
 
 _ARRAY_IDS = {"Ip": 1, "Iz": 2, "W": 3, "X": 4}
