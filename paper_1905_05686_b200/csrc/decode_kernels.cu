@@ -219,7 +219,7 @@ __device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane)
 
 // SEGQ = 128-column quads per run of columns that lies inside one tile (8: the whole block).
 template <int SEGQ>
-__global__ void __launch_bounds__(DEC_THREADS)
+__global__ void __launch_bounds__(DEC_THREADS, SEGQ <= 2 ? 8 : 4)
 decode_planes_wide_kernel(Geo g, int row_bands_per_tile, int rows_per_block,
                           const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz,
                           uint32_t *__restrict__ mask)
@@ -264,13 +264,14 @@ decode_planes_wide_kernel(Geo g, int row_bands_per_tile, int rows_per_block,
     // ---- one thread per mask row; per run of quads inside one tile, OR the planes its Ip word selects
     const bool vec = (g.pitch & 3) == 0;
     for (int i = i_first; i < min(i_end, (band + 1) * rows_per_block); i += DEC_THREADS) {
-        uint4 acc[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) acc[q] = make_uint4(0, 0, 0, 0);
+        uint32_t *dst = mask + (long long)(tr * g.tm + i) * g.pitch + gw0;
 #pragma unroll
         for (int seg = 0; seg < 8 / SEGQ; ++seg) {
             const int gw = gw0 + seg * SEGQ * 4;                // first mask word of the run
             if (gw >= g.pitch) break;
+            uint4 acc[SEGQ];                                    // the run's index bits of this row
+#pragma unroll
+            for (int q = 0; q < SEGQ; ++q) acc[q] = make_uint4(0, 0, 0, 0);
             const int tc = gw / words_in_tile;
             const uint32_t *ipw = ip + (((long long)tr * g.gc + tc) * g.tm + i) * g.kw;
             auto or_planes = [&](uint32_t x, int lb) {
@@ -282,7 +283,7 @@ decode_planes_wide_kernel(Geo g, int row_bands_per_tile, int rows_per_block,
 #pragma unroll
                     for (int q = 0; q < SEGQ; ++q) {
                         const uint4 v = src[q];
-                        uint4 &a = acc[seg * SEGQ + q];
+                        uint4 &a = acc[q];
                         a.x |= v.x; a.y |= v.y; a.z |= v.z; a.w |= v.w;
                     }
                 }
@@ -293,16 +294,17 @@ decode_planes_wide_kernel(Geo g, int row_bands_per_tile, int rows_per_block,
             } else {
                 for (int lb = 0; lb < g.kw; ++lb) or_planes(__ldg(ipw + lb), lb);
             }
-        }
-        uint32_t *dst = mask + (long long)(tr * g.tm + i) * g.pitch + gw0;
+            // store the run; the thread's runs together fill one 128-byte line of its mask row
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int nw = g.pitch - gw0 - q * 4;                // words of this quad that exist in the row
-            if (nw >= 4 && vec) {
-                reinterpret_cast<uint4 *>(dst)[q] = acc[q];
-            } else if (nw > 0) {
-                const uint32_t v[4] = {acc[q].x, acc[q].y, acc[q].z, acc[q].w};
-                for (int e = 0; e < min(nw, 4); ++e) dst[q * 4 + e] = v[e];
+            for (int q = 0; q < SEGQ; ++q) {
+                const int w = seg * SEGQ * 4 + q * 4;           // word inside the block
+                const int nw = g.pitch - gw0 - w;               // words of this quad that exist in the row
+                if (nw >= 4 && vec) {
+                    *reinterpret_cast<uint4 *>(dst + w) = acc[q];
+                } else if (nw > 0) {
+                    const uint32_t v[4] = {acc[q].x, acc[q].y, acc[q].z, acc[q].w};
+                    for (int e = 0; e < min(nw, 4); ++e) dst[w + e] = v[e];
+                }
             }
         }
     }
