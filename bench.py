@@ -28,6 +28,9 @@ from paper_1905_05686_b200 import synth  # noqa: E402
 METRIC = "fused decode+masked-GEMM TFLOP/s and effective HBM GB/s vs roofline"
 DEFAULT_WORKLOAD = "ffn_16384x4096"
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu capture
+# summarised under profiles/ (null for workloads without a capture of the current kernel)
+NCU_TRAFFIC_BYTES = {("ffn_16384x4096", 4096): 353532160}
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -324,7 +327,7 @@ def run_ours(args):
     else:
         achieved = work_flops / (kernel_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                    "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get((args.workload, batch)),
                     "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
     roofline["peak_source"] = "of " + peaks["source"]
     roofline["kernel_ms"] = kernel_ms

@@ -92,6 +92,8 @@ RAGGED = [
     (260, 300, 130, 150, 145),    # the paper's LSTM rank
     (300, 520, 300, 520, 256),
     (70, 4100, 64, 4096, 3),
+    (300, 640, 100, 128, 16),     # 128-column tiles: every 128-column run of a mask row has its own tile
+    (1300, 1536, 1300, 768, 40),  # 768-column tiles (runs of two quads), more than 1024 rows per tile
 ]
 
 
