@@ -207,6 +207,48 @@ __host__ __device__ constexpr uint32_t make_idesc(int bn, int m = TC_BM)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// 16-byte asynchronous copy global -> shared; bytes beyond `valid` (0..16) are written as zero.
+__device__ __forceinline__ void cp_async_16(void *dst_smem, const void *src, int valid)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(valid) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// Stage the factor words of one panel: the Iz words of its `pw32` columns (first column c0, tile row tr)
+// and the Ip words of the block's 128 rows (first row o0).  Words outside the tile are written as zero.
+// Asynchronous copies (one commit group); the caller waits for them.  dt = 0 .. nthreads-1.
+__device__ __forceinline__ void stage_panel_factors(const Geo &g, const uint32_t *__restrict__ ip,
+                                                    const uint32_t *__restrict__ iz, uint32_t *iz_stage,
+                                                    uint32_t *ip_stage, int pw32, int c0, int o0, int dt, int nthreads)
+{
+    const int zwords = pw32 * g.kw, xwords = TC_BM * g.kw;
+    if (o0 >= g.rows) {                                  // a block without rows of W (second CTA of a ragged pair)
+        for (int q = dt; q < zwords; q += nthreads) iz_stage[q] = 0u;
+        for (int q = dt; q < xwords; q += nthreads) ip_stage[q] = 0u;
+        return;
+    }
+    // 16-byte copies need 16-byte aligned sources: tile bases are, unless a tile holds an odd word count
+    const bool z_vec = ((g.tn * g.kw) & 3) == 0, x_vec = ((g.tm * g.kw) & 3) == 0;
+    const int tr = o0 / g.tm, i0 = o0 - tr * g.tm;       // tile row, first row of the block inside its tile
+    const int tc = c0 / g.tn, j0 = c0 - tc * g.tn;       // tile column, first column of the panel inside its tile
+    const size_t tile = (size_t)tr * g.gc + tc;
+    const uint32_t *zsrc = iz + (tile * g.tn + j0) * g.kw;
+    const uint32_t *xsrc = ip + (tile * g.tm + i0) * g.kw;
+    const int zvalid = (g.tn - j0) * g.kw, xvalid = (g.tm - i0) * g.kw;   // words that exist in the tile
+    for (int q = dt * 4; q < zwords; q += nthreads * 4) {
+        const int n = min(4, max(0, zvalid - q));
+        if (z_vec) cp_async_16(iz_stage + q, zsrc + (n > 0 ? q : 0), n * 4);
+        else for (int e = 0; e < 4; ++e) iz_stage[q + e] = e < n ? __ldg(zsrc + q + e) : 0u;
+    }
+    for (int q = dt * 4; q < xwords; q += nthreads * 4) {
+        const int n = min(4, max(0, xvalid - q));
+        if (x_vec) cp_async_16(ip_stage + q, xsrc + (n > 0 ? q : 0), n * 4);
+        else for (int e = 0; e < 4; ++e) ip_stage[q + e] = e < n ? __ldg(xsrc + q + e) : 0u;
+    }
+    cp_async_commit();
+}
+
 // Shared-memory bookkeeping that follows the operand stages.
 struct TcCtl {
     uint64_t full[8];        // TMA copies of a stage have landed
@@ -277,14 +319,6 @@ __device__ __forceinline__ void transpose32_x4(uint32_t (&x)[4], int lane)
     }
 }
 
-// 16-byte asynchronous copy global -> shared; bytes beyond `valid` (0..16) are written as zero.
-__device__ __forceinline__ void cp_async_16(void *dst_smem, const void *src, int valid)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(valid) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-
 // Zero the pruned halves of the eight bf16 values of one 16-byte chunk.  `bits` holds the index
 // bits of the row's 32 columns in the permuted order above; chunk j uses groups 2j and 2j+1.
 __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
@@ -345,6 +379,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     const int kb_end = min(nkb_total, kb_begin + kb_per_split);
     const int nkb = kb_end - kb_begin;                   // >= 1 by construction of the grid
 
+    // Long-latency requests first: the decoder warps ask for the factor words of their first panel, one
+    // thread warms the TMA descriptors; both overlap the barrier and tensor-memory set-up below.
+    if (warp >= 2 + TC_MASK_WARPS)
+        stage_panel_factors(g, ip, iz, iz_stage, ip_stage, PW * 32, kb_begin * TC_BK, o0,
+                            threadIdx.x - (2 + TC_MASK_WARPS) * 32, TC_DECODE_WARPS * 32);
+    if (threadIdx.x == 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&w_map) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&ctl->full[s], 1);
@@ -449,32 +492,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         // 16-byte copies need 16-byte aligned sources: tile bases are, unless a tile holds an odd word count
         const bool z_vec = ((g.tn * g.kw) & 3) == 0, x_vec = ((g.tm * g.kw) & 3) == 0;
 
-        // Stage the factor words of panel P: Iz words of its PW*32 columns, Ip words of the 128 rows.
-        // Words outside the tile are written as zero.  Asynchronous copies; the caller waits for them.
         auto stage_factors = [&](int P) {
-            if (P >= npanels) return;
-            if (o0 >= g.rows) {                          // a block without rows of W (second CTA of a ragged pair)
-                for (int q = dt; q < zwords; q += TC_DECODE_WARPS * 32) iz_stage[q] = 0u;
-                for (int q = dt; q < xwords; q += TC_DECODE_WARPS * 32) ip_stage[q] = 0u;
-                return;
-            }
-            const int c0 = (kb_begin + P * KBP) * TC_BK;            // first column of the panel
-            const int tc = c0 / g.tn, j0 = c0 - tc * g.tn;           // ... its tile column, column inside the tile
-            const size_t tile = (size_t)tr * g.gc + tc;
-            const uint32_t *zsrc = iz + (tile * g.tn + j0) * g.kw;
-            const uint32_t *xsrc = ip + (tile * g.tm + i0) * g.kw;
-            const int zvalid = (g.tn - j0) * g.kw, xvalid = (g.tm - i0) * g.kw;   // words that exist in the tile
-            for (int q = dt * 4; q < zwords; q += TC_DECODE_WARPS * 32 * 4) {
-                const int n = min(4, max(0, zvalid - q));
-                if (z_vec) cp_async_16(iz_stage + q, zsrc + (n > 0 ? q : 0), n * 4);
-                else for (int e = 0; e < 4; ++e) iz_stage[q + e] = e < n ? __ldg(zsrc + q + e) : 0u;
-            }
-            for (int q = dt * 4; q < xwords; q += TC_DECODE_WARPS * 32 * 4) {
-                const int n = min(4, max(0, xvalid - q));
-                if (x_vec) cp_async_16(ip_stage + q, xsrc + (n > 0 ? q : 0), n * 4);
-                else for (int e = 0; e < 4; ++e) ip_stage[q + e] = e < n ? __ldg(xsrc + q + e) : 0u;
-            }
-            cp_async_commit();
+            if (P < npanels)
+                stage_panel_factors(g, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + P * KBP) * TC_BK, o0, dt, TC_DECODE_WARPS * 32);
         };
 
         uint32_t dsync_parity = 0;
@@ -486,7 +506,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             dsync_parity ^= 1;
         };
 
-        stage_factors(0);
+        // (panel 0 was requested at kernel entry)
         for (int P = 0; P < npanels && ok; ++P) {
             const int buf = P & 1;
             uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
