@@ -335,7 +335,10 @@ lrbi_status launch_decode_planes(const Geo &g, const uint32_t *ip, const uint32_
                                  cudaStream_t s)
 {
     if (!decode_planes_supported(g)) return LRBI_ERR_UNSUPPORTED;
-    if (decode_planes_wide_supported(g)) return launch_decode_planes_wide(g, ip, iz, mask, s);
+    // the wide variant wants enough 1024-column blocks to fill the chip; a small mask is better served by
+    // the many small blocks of the 256-column variant
+    const long long wide_blocks = (long long)((g.pitch + WIDE_WORDS - 1) / WIDE_WORDS) * g.gr * ((g.tm + 1023) / 1024);
+    if (decode_planes_wide_supported(g) && wide_blocks >= 256) return launch_decode_planes_wide(g, ip, iz, mask, s);
     const int cbpt = ((g.tn >> 5) + DEC_WORDS - 1) / DEC_WORDS;
     const int rbpt = (g.tm + PLANES_ROWS_PER_BLOCK - 1) / PLANES_ROWS_PER_BLOCK;
     dim3 grid((unsigned)(g.gc * cbpt), (unsigned)(g.gr * rbpt));
