@@ -75,7 +75,8 @@ enum {
     LRBI_ALGO_GEMV = 2,      /* small batch, bandwidth-bound, CUDA-core FMA                    */
     LRBI_ALGO_TENSOR = 3,    /* tcgen05 MMA with TMEM accumulators                             */
     LRBI_ALGO_DECODE_BALLOT = 4, /* decode: one __ballot_sync per 32-bit mask word             */
-    LRBI_ALGO_DECODE_PLANES = 5  /* decode: ballot-transposed Iz bit-planes, OR per 32 columns */
+    LRBI_ALGO_DECODE_PLANES = 5, /* decode: Iz transposed into bit-planes, OR per 32 columns (variant by size) */
+    LRBI_ALGO_DECODE_PLANES_WIDE = 6 /* decode: the 1024-column bit-plane variant, whatever the mask size */
 };
 
 /* Element counts of the packed arrays for a layout (0 if the layout is invalid). */
@@ -88,8 +89,9 @@ LRBI_API size_t lrbi_mask_words(const lrbi_layout *layout);      /* rows*ceil(co
  *   ip, iz    device, packed factors as above (read only)
  *   mask_out  device, rows x ceil(cols/32) uint32, row-major; bit (c % 32) of word c / 32
  *             of row r is Ia[r][c]; bits beyond `cols` in the last word of a row are 0.
- *   algo      LRBI_ALGO_AUTO, LRBI_ALGO_DECODE_BALLOT or LRBI_ALGO_DECODE_PLANES
- *             (PLANES needs tile_cols % 32 == 0, else LRBI_ERR_UNSUPPORTED)
+ *   algo      LRBI_ALGO_AUTO, LRBI_ALGO_DECODE_BALLOT, LRBI_ALGO_DECODE_PLANES (needs
+ *             tile_cols % 32 == 0) or LRBI_ALGO_DECODE_PLANES_WIDE (needs tile_cols % 128 == 0 and
+ *             rank <= 256); a variant that does not cover the layout returns LRBI_ERR_UNSUPPORTED
  * Every word of mask_out is written; nothing else is.
  */
 LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t *ip, const uint32_t *iz,

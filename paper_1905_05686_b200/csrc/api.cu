@@ -85,6 +85,7 @@ lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t *ip, cons
                                           : launch_decode_ballot(g, ip, iz, mask_out, s);
     case LRBI_ALGO_DECODE_BALLOT: return launch_decode_ballot(g, ip, iz, mask_out, s);
     case LRBI_ALGO_DECODE_PLANES: return launch_decode_planes(g, ip, iz, mask_out, s);
+    case LRBI_ALGO_DECODE_PLANES_WIDE: return launch_decode_planes_wide(g, ip, iz, mask_out, s);
     default: return LRBI_ERR_INVALID_ARG;
     }
 }

@@ -312,9 +312,10 @@ decode_planes_wide_kernel(Geo g, int row_bands_per_tile, int rows_per_block,
 
 static bool decode_planes_wide_supported(const Geo &g) { return (g.tn % 128) == 0 && g.k <= WIDE_MAX_RANK; }
 
-static lrbi_status launch_decode_planes_wide(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask,
-                                             cudaStream_t s)
+lrbi_status launch_decode_planes_wide(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask,
+                                      cudaStream_t s)
 {
+    if (!decode_planes_wide_supported(g)) return LRBI_ERR_UNSUPPORTED;
     const int rows_per_block = g.tm >= 1024 ? 1024 : (g.tm + DEC_THREADS - 1) / DEC_THREADS * DEC_THREADS;
     const int rbpt = (g.tm + rows_per_block - 1) / rows_per_block;
     dim3 grid((unsigned)((g.pitch + WIDE_WORDS - 1) / WIDE_WORDS), (unsigned)(g.gr * rbpt));

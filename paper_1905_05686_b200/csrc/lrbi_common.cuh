@@ -63,6 +63,7 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
 lrbi_status launch_decode_ballot(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
 lrbi_status launch_decode_planes(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
 bool decode_planes_supported(const Geo &g);
+lrbi_status launch_decode_planes_wide(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
 
 lrbi_status launch_gemm_generic(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                                 const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);

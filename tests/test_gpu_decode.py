@@ -50,7 +50,8 @@ ALGOS = ["auto", "ballot", "planes"]
 
 def _algo(name):
     b = _b()
-    return {"auto": b.ALGO_AUTO, "ballot": b.ALGO_DECODE_BALLOT, "planes": b.ALGO_DECODE_PLANES}[name]
+    return {"auto": b.ALGO_AUTO, "ballot": b.ALGO_DECODE_BALLOT, "planes": b.ALGO_DECODE_PLANES,
+            "wide": b.ALGO_DECODE_PLANES_WIDE}[name]
 
 
 @pytest.mark.parametrize("algo", ALGOS)
@@ -110,6 +111,14 @@ def test_ragged_shapes_planes(shape):
     check(synth.Layer("rag", rows, cols, tm, tn, k, 0.2), _algo("planes"))
 
 
+@pytest.mark.parametrize("shape", [s for s in RAGGED if s[3] % 128 == 0 and s[4] <= 256] +
+                         [(4096, 4096, 256, 256, 8), (2100, 3072, 1050, 1024, 64), (600, 2304, 128, 256, 16)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_ragged_shapes_planes_wide(shape):
+    rows, cols, tm, tn, k = shape
+    check(synth.Layer("rag", rows, cols, tm, tn, k, 0.2), _algo("wide"))
+
+
 def test_planes_refuses_unaligned_tiles():
     b = _b()
     L = synth.Layer("rag", 37, 45, 16, 20, 7, 0.2)
@@ -119,9 +128,9 @@ def test_planes_refuses_unaligned_tiles():
     assert e.value.code == b.ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("algo", ["ballot", "planes"])
+@pytest.mark.parametrize("algo", ["ballot", "planes", "wide"])
 def test_degenerate_factors(algo):
-    L = synth.Layer("deg", 96, 160, 32, 32, 5, 0.2)
+    L = synth.Layer("deg", 96, 160, 32, 32, 5, 0.2) if algo != "wide" else synth.Layer("deg", 96, 640, 32, 128, 5, 0.2)
     for p in (0.0, 1.0):
         check(L, _algo(algo), p=p)                              # empty and full masks
 
