@@ -30,7 +30,10 @@ DEFAULT_WORKLOAD = "ffn_16384x4096"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu capture
 # summarised under profiles/ (null for workloads without a capture of the current kernel)
-NCU_TRAFFIC_BYTES = {("ffn_16384x4096", 4096): 353532160}
+NCU_TRAFFIC_BYTES = {("ffn_16384x4096", 4096): 336644352,      # gemm_tc_kernel<256, 8, pair>
+                     ("decode_32768", 0): 136190000,            # decode_planes_wide_kernel<2>
+                     ("alexnet_fc", 1): 77350000,               # gemv_kernel<1, 8, 1>
+                     ("alexnet_fc", 16): 78600000}              # gemm_tc_kernel<16, 8> (the reduce kernel adds 2.4 MB)
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -323,7 +326,7 @@ def run_ours(args):
     if decode_only or B.masked_gemm_choice(layer, batch) == B.ALGO_GEMV or work_flops / work_bytes < peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9):
         achieved = work_bytes / (kernel_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None}
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((args.workload, batch))}
     else:
         achieved = work_flops / (kernel_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
