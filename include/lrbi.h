@@ -76,7 +76,8 @@ enum {
     LRBI_ALGO_TENSOR = 3,    /* tcgen05 MMA with TMEM accumulators                             */
     LRBI_ALGO_DECODE_BALLOT = 4, /* decode: one __ballot_sync per 32-bit mask word             */
     LRBI_ALGO_DECODE_PLANES = 5, /* decode: Iz transposed into bit-planes, OR per 32 columns (variant by size) */
-    LRBI_ALGO_DECODE_PLANES_WIDE = 6 /* decode: the 1024-column bit-plane variant, whatever the mask size */
+    LRBI_ALGO_DECODE_PLANES_WIDE = 6, /* decode: the 1024-column bit-plane variant, whatever the mask size */
+    LRBI_ALGO_STREAM = 7     /* batch <= 32, bandwidth-bound, warp-level tensor-core MMAs              */
 };
 
 /* Element counts of the packed arrays for a layout (0 if the layout is invalid). */
@@ -105,7 +106,7 @@ LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t 
  *   W      device, bf16 bit patterns, [rows][cols] row-major
  *   X      device, bf16 bit patterns, [batch][cols] row-major
  *   Y      device, [batch][rows] row-major, bf16 (round to nearest even) or fp32 per y_dtype
- *   algo   LRBI_ALGO_AUTO, _GENERIC, _GEMV (batch <= 8) or _TENSOR; a kernel that does not
+ *   algo   LRBI_ALGO_AUTO, _GENERIC, _GEMV (batch <= 8), _STREAM (batch <= 32) or _TENSOR; a kernel that does not
  *          cover the shape returns LRBI_ERR_UNSUPPORTED and launches nothing.
  * The tensor-core path may split the reduction over several thread blocks; it then keeps
  * fp32 partial sums in a library-owned device buffer that grows (cudaMalloc) on the first

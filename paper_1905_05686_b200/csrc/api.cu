@@ -42,8 +42,10 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 static int choose_gemm(const Geo &g, int batch)
 {
-    // measured on B200 (4096 x 9216 layer): the CUDA-core kernel wins up to batch 4 (23 us at batch 1 against
-    // 32 us); from batch 8 on its fp32 FMAs cost more than the tensor-core kernel's fixed latencies
+    // measured on B200 (4096 x 9216 layer, microseconds, CUDA-core GEMV / warp-MMA stream / tcgen05):
+    // batch 1: 22 / 28 / 30; batch 2: 31 / 28 / 30; batch 4: 29 / 27 / 30; batch 8: 64 / 29 / 30; batch 16: - / 31 / 30
+    if (batch == 1 && gemv_supported(g, batch)) return LRBI_ALGO_GEMV;
+    if (batch <= 8 && stream_mma_supported(g, batch)) return LRBI_ALGO_STREAM;
     if (batch <= 4 && gemv_supported(g, batch)) return LRBI_ALGO_GEMV;
     if (gemm_tc_supported(g, batch)) return LRBI_ALGO_TENSOR;
     return LRBI_ALGO_GENERIC;
@@ -111,6 +113,7 @@ lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const
     switch (algo) {
     case LRBI_ALGO_GENERIC: return launch_gemm_generic(g, W, ip, iz, X, batch, Y, y_dtype, s);
     case LRBI_ALGO_GEMV: return launch_gemv(g, W, ip, iz, X, batch, Y, y_dtype, s);
+    case LRBI_ALGO_STREAM: return launch_stream_mma(g, W, ip, iz, X, batch, Y, y_dtype, s);
     case LRBI_ALGO_TENSOR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s);
     default: return LRBI_ERR_INVALID_ARG;
     }

@@ -70,6 +70,9 @@ lrbi_status launch_gemm_generic(const Geo &g, const uint16_t *W, const uint32_t 
 bool gemv_supported(const Geo &g, int batch);
 lrbi_status launch_gemv(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                         const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+bool stream_mma_supported(const Geo &g, int batch);
+lrbi_status launch_stream_mma(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                              const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 bool gemm_tc_supported(const Geo &g, int batch);
 // `partials` == nullptr lets the launcher use the library-owned buffer when it splits K.
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,

@@ -100,11 +100,11 @@ def test_small_shapes_every_kernel_that_covers_them(shape):
     c = Case(L, batch)
     want = c.oracle_full()
     tried = 0
-    for algo in (b.ALGO_GENERIC, b.ALGO_GEMV, b.ALGO_TENSOR, b.ALGO_AUTO):
+    for algo in (b.ALGO_GENERIC, b.ALGO_GEMV, b.ALGO_STREAM, b.ALGO_TENSOR, b.ALGO_AUTO):
         try:
             got = c.run(algo)
         except b.LrbiError as e:
-            assert e.code == b.ERR_UNSUPPORTED and algo in (b.ALGO_GEMV, b.ALGO_TENSOR)
+            assert e.code == b.ERR_UNSUPPORTED and algo in (b.ALGO_GEMV, b.ALGO_STREAM, b.ALGO_TENSOR)
             continue
         tried += 1
         assert rel_fro(got, want) <= TOL, (b.ALGO_NAMES[algo], rel_fro(got, want))
@@ -139,6 +139,31 @@ def test_tensor_core_kernel(shape):
     got = c.run(b.ALGO_TENSOR)
     assert rel_fro(got, want) <= TOL, rel_fro(got, want)
     got32 = c.run(b.ALGO_TENSOR, torch.float32)
+    assert rel_fro(got32, want) <= TOL_F32, rel_fro(got32, want)
+
+
+STREAM_SHAPES = [
+    # rows, cols, tm, tn, k, batch
+    (16, 32, 16, 32, 4, 1),
+    (500, 800, 500, 800, 16, 7),          # ragged rows, 800 = 25 steps of 32
+    (500, 808, 500, 808, 16, 9),          # last step has columns in one lane group only
+    (384, 1024, 128, 256, 64, 16),
+    (640, 1088, 128, 64, 33, 17),
+    (1024, 4096, 512, 1024, 64, 32),
+    (272, 2304, 16, 256, 16, 5),
+]
+
+
+@pytest.mark.parametrize("shape", STREAM_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_stream_kernel(shape):
+    b = _b()
+    rows, cols, tm, tn, k, batch = shape
+    L = synth.Layer("stream", rows, cols, tm, tn, k, 0.25, 0.05)
+    c = Case(L, batch)
+    want = c.oracle_full()
+    got = c.run(b.ALGO_STREAM)
+    assert rel_fro(got, want) <= TOL, rel_fro(got, want)
+    got32 = c.run(b.ALGO_STREAM, torch.float32)
     assert rel_fro(got32, want) <= TOL_F32, rel_fro(got32, want)
 
 
