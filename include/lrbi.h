@@ -50,7 +50,7 @@ extern "C" {
 typedef enum {
     LRBI_OK = 0,
     LRBI_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer          */
-    LRBI_ERR_UNSUPPORTED = 2, /* a shape, dtype or kernel choice this build does not cover     */
+    LRBI_ERR_UNSUPPORTED = 2, /* a shape, dtype or kernel choice this library does not cover   */
     LRBI_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed (see lrbi_last_cuda_error)  */
     LRBI_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up (see lrbi_device_status)   */
     LRBI_ERR_TOO_LARGE = 5    /* the problem needs more fixed scratch than the library carries   */
