@@ -636,16 +636,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             tc_fence_after();
             // All MMAs have completed, so the operand stages are free: reuse them to transpose the
             // accumulator (lane = output feature) into rows of Y (contiguous output features).  The
-            // accumulator goes through in passes of at most 64 batch columns (128 x 64 x 4 bytes = 32 KB,
-            // which every stage configuration has room for).
+            // accumulator goes through in as few passes as the stage memory allows (all 256 columns at once
+            // for bf16 output in pair mode, halves for fp32).
             const bool out32 = partials != nullptr || y_dtype == LRBI_Y_F32;
             const int esz = out32 ? 4 : 2;
             const int quad = warp & 3;                   // tensor-memory lanes this warp may read
             const int half = mw >> 2;                    // which half of a pass's columns
             const int ol = quad * 32 + lane;             // output feature inside the block
-            constexpr int PASS = BN < 64 ? BN : 64;      // batch columns per pass
-            constexpr int COLS_PER_WARP = PASS / 2 < 16 ? 16 : PASS / 2;
-            constexpr int NCHUNK = COLS_PER_WARP / 16;
+            const int room = stages * (TC_A_STAGE_BYTES + B_STAGE_BYTES) / (TC_BM * esz);   // columns the stages can hold
+            const int PASS = BN < 32 ? BN : min(BN, room & ~31);                            // batch columns per pass
+            const int COLS_PER_WARP = PASS / 2 < 16 ? 16 : PASS / 2;
+            const int NCHUNK = COLS_PER_WARP / 16;
             uint8_t *dst_base = partials ? reinterpret_cast<uint8_t *>(partials + (long long)blockIdx.z * batch * g.rows)
                                          : reinterpret_cast<uint8_t *>(Y);
             const int row_bytes = TC_BM * esz;           // one batch row of the block
