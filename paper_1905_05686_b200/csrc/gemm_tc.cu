@@ -644,7 +644,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             const int half = mw >> 2;                    // which half of a pass's columns
             const int ol = quad * 32 + lane;             // output feature inside the block
             const int room = stages * (TC_A_STAGE_BYTES + B_STAGE_BYTES) / (TC_BM * esz);   // columns the stages can hold
-            const int PASS = BN < 32 ? BN : min(BN, room & ~31);                            // batch columns per pass
+            int PASS = BN;                               // batch columns per pass: BN, BN/2, ... down to 32 (or BN if smaller)
+            while (PASS > 32 && PASS > room) PASS >>= 1;                                    // always a divisor of BN
             const int COLS_PER_WARP = PASS / 2 < 16 ? 16 : PASS / 2;
             const int NCHUNK = COLS_PER_WARP / 16;
             uint8_t *dst_base = partials ? reinterpret_cast<uint8_t *>(partials + (long long)blockIdx.z * batch * g.rows)
