@@ -353,7 +353,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     constexpr int B_STAGE_BYTES = B_ROWS * TC_BK * 2;
     constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
     constexpr int KBP = PW / 2;                          // K blocks per panel
-    constexpr int PWH = PW / 2;                          // index words a thread decodes per row
     uint8_t *a_base = smem;
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
     constexpr int PWS = PW == 8 ? 12 : PW;               // words between planes (padded: conflict-free 16-byte reads)
@@ -488,9 +487,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         const int bit_col = column_of_bit(lane);        // column (0..31) this lane stands for in a transpose
         const int npairs = g.kw * PW;                   // (32-plane block, index word) pairs of a panel
         const int npanels = (nkb + KBP - 1) / KBP;
-        const int zwords = PW * 32 * g.kw, xwords = TC_BM * g.kw;   // factor words of a panel / of the 128 rows
-        // 16-byte copies need 16-byte aligned sources: tile bases are, unless a tile holds an odd word count
-        const bool z_vec = ((g.tn * g.kw) & 3) == 0, x_vec = ((g.tm * g.kw) & 3) == 0;
 
         auto stage_factors = [&](int P) {
             if (P < npanels)
