@@ -30,10 +30,10 @@ DEFAULT_WORKLOAD = "ffn_16384x4096"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu capture
 # summarised under profiles/ (null for workloads without a capture of the current kernel)
-NCU_TRAFFIC_BYTES = {("ffn_16384x4096", 4096): 344390000,      # gemm_tc_kernel<256, 8, pair>
-                     ("decode_32768", 0): 136190000,            # decode_planes_wide_kernel<2>
-                     ("alexnet_fc", 1): 77350000,               # gemv_kernel<1, 8, 1>
-                     ("alexnet_fc", 16): 78600000}              # gemm_tc_kernel<16, 8> (the reduce kernel adds 2.4 MB)
+NCU_TRAFFIC_BYTES = {}
+# The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
+OTHER_WORKLOADS = [("lenet_fc1", 32), ("decode_4096", 0), ("decode_32768", 0), ("alexnet_fc", 1), ("alexnet_fc", 16),
+                   ("alexnet_fc", 128), ("conv3x3_256", 12544)]
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -150,12 +150,12 @@ def oracle_sample_run(layer: synth.Layer, batch: int, target_s: float = 15.0, ro
         t1 = max(time.perf_counter() - t0, 1e-4)
         rows_sample = int(max(1, min(batch, (target_s - t_dec) / t1)))
     t0 = time.perf_counter()
-    oracle.masked_gemm(Wb, M, Xb[:rows_sample])
+    y_ref = oracle.masked_gemm(Wb, M, Xb[:rows_sample])
     t_gemm = time.perf_counter() - t0
     flops = dense_flops(layer, rows_sample)
     text = "full index decode (%d x %d) + masked product for the first %d of %d batch rows" % (
         layer.rows, layer.cols, rows_sample, batch)
-    return flops, t_dec + t_gemm, text, rows_sample
+    return flops, t_dec + t_gemm, text, rows_sample, y_ref
 
 
 def run_reference(args):
@@ -174,7 +174,7 @@ def run_reference(args):
     flops = 0
     text = ""
     for i in range(warmup + steps):
-        flops, sec, text, rows_sample = oracle_sample_run(layer, batch, per_step, rows_sample)
+        flops, sec, text, rows_sample, _ = oracle_sample_run(layer, batch, per_step, rows_sample)
         if i >= warmup:
             times.append(sec)
     ms = 1e3 * float(np.mean(times))
@@ -194,6 +194,61 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------ GPU arm
+def roofline_of(workload, batch, work_bytes, work_flops, kernel_ms, peaks):
+    """Roofline of one launch: the bound is the one that needs the longer time at the measured peaks."""
+    t_hbm = work_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_tc = work_flops / (peaks["bf16_tflops"] * 1e12)
+    if t_hbm >= t_tc:
+        achieved = work_bytes / (kernel_ms * 1e-3) / 1e9
+        r = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"]}
+    else:
+        achieved = work_flops / (kernel_ms * 1e-3) / 1e12
+        r = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+             "frac": achieved / peaks["bf16_tflops"], "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
+    r["traffic"] = NCU_TRAFFIC_BYTES.get((workload, batch))
+    r["peak_source"] = "of " + peaks["source"]
+    r["kernel_ms"] = kernel_ms
+    return r
+
+
+def kernel_label(B, layer, batch):
+    if not batch:
+        return "decode"
+    plan = B.masked_gemm_plan(layer, batch)
+    name = B.ALGO_NAMES[plan.algo]
+    if plan.algo == B.ALGO_TENSOR:
+        name += " tile%d%s panel%d splits%d stages%d" % (plan.batch_tile, " pair" if plan.cta_pair else "", plan.panel_columns,
+                                                          plan.k_splits, plan.stages)
+    return name
+
+
+def setup_workload(B, workload, batch, rank=0):
+    """Device buffers and the step function of one workload.  Returns a dict."""
+    import torch
+
+    layer = synth.CONFIGS[workload]
+    decode_only = not layer.batches
+    batch = 0 if decode_only else (batch or layer.batches[-1])
+    Ip, Iz = synth.make_factors(layer)
+    ipw, izw = synth.pack_ip(Ip), synth.pack_iz(Iz)
+    ip, iz = B.to_device_words(ipw), B.to_device_words(izw)
+    w = {"layer": layer, "batch": batch, "decode_only": decode_only, "Ip": Ip, "Iz": Iz, "ipw": ipw, "izw": izw}
+    if decode_only:
+        out = torch.empty((layer.rows, (layer.cols + 31) // 32), dtype=torch.int32, device="cuda")
+        w.update(step=lambda: B.lrbi_decode_mask(layer, ip, iz, out), out=out,
+                 work_bytes=decode_bytes(layer), work_flops=0)
+    else:
+        Wb = synth.make_weights(layer)
+        xlayer = synth.Layer(**{**layer.__dict__, "seed": rank_seed(layer.seed, rank)})
+        Xb = synth.make_activations(xlayer, batch)
+        W, X = B.to_device_bf16(Wb), B.to_device_bf16(Xb)
+        Y = torch.empty((batch, layer.rows), dtype=torch.bfloat16, device="cuda")
+        w.update(step=lambda: B.lrbi_masked_gemm(layer, W, ip, iz, X, Y=Y), out=Y, Wb=Wb, Xb=Xb,
+                 work_bytes=algorithmic_bytes(layer, batch), work_flops=dense_flops(layer, batch))
+    w["keep"] = (ip, iz)
+    return w
+
+
 def time_calls(fn, n, warmup, flush_buf=None, stream=None):
     """Per-call device times (ms) with CUDA events on the launching stream."""
     import torch
@@ -229,26 +284,13 @@ def run_ours(args):
 
     B.lib()
     peaks = load_peaks()
-    layer = synth.CONFIGS[args.workload]
-    decode_only = not layer.batches
-    batch = 0 if decode_only else (args.batch or layer.batches[-1])
-
-    Ip, Iz = synth.make_factors(layer)
-    ipw, izw = synth.pack_ip(Ip), synth.pack_iz(Iz)
-    ip, iz = B.to_device_words(ipw), B.to_device_words(izw)
+    wl = setup_workload(B, args.workload, args.batch, rank)
+    layer, batch, decode_only, step = wl["layer"], wl["batch"], wl["decode_only"], wl["step"]
+    work_bytes, work_flops = wl["work_bytes"], wl["work_flops"]
+    Ip, Iz, ipw, izw = wl["Ip"], wl["Iz"], wl["ipw"], wl["izw"]
+    if not decode_only:
+        Wb, Xb, Y = wl["Wb"], wl["Xb"], wl["out"]
     flush = None
-    if decode_only:
-        out = torch.empty((layer.rows, (layer.cols + 31) // 32), dtype=torch.int32, device="cuda")
-        step = lambda: B.lrbi_decode_mask(layer, ip, iz, out)
-        work_bytes, work_flops = decode_bytes(layer), 0
-    else:
-        Wb = synth.make_weights(layer)
-        xlayer = synth.Layer(**{**layer.__dict__, "seed": rank_seed(layer.seed, rank)})
-        Xb = synth.make_activations(xlayer, batch)
-        W, X = B.to_device_bf16(Wb), B.to_device_bf16(Xb)
-        Y = torch.empty((batch, layer.rows), dtype=torch.bfloat16, device="cuda")
-        step = lambda: B.lrbi_masked_gemm(layer, W, ip, iz, X, Y=Y)
-        work_bytes, work_flops = algorithmic_bytes(layer, batch), dense_flops(layer, batch)
     footprint = work_bytes
     if footprint <= L2_BYTES:
         flush = torch.zeros(256 * 1024 * 1024 // 4, dtype=torch.int32, device="cuda")
@@ -328,33 +370,57 @@ def run_ours(args):
     # ---- roofline of the dominant kernel (one launch per step for this workload)
     launches_per_step = launches / args.steps
     kernel_ms = float(np.mean(per_step))
-    if decode_only or B.masked_gemm_choice(layer, batch) == B.ALGO_GEMV or work_flops / work_bytes < peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9):
-        achieved = work_bytes / (kernel_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((args.workload, batch))}
-    else:
-        achieved = work_flops / (kernel_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get((args.workload, batch)),
-                    "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
-    roofline["peak_source"] = "of " + peaks["source"]
-    roofline["kernel_ms"] = kernel_ms
+    roofline = roofline_of(args.workload, batch, work_bytes, work_flops, kernel_ms, peaks)
     roofline["launches_per_step"] = launches_per_step
 
     # ---- CPU oracle on a bounded sample of the same workload
-    cpu = None
+    cpu, parity = None, None
     if not args.no_cpu_baseline:
         import oracle
         if decode_only:
             t0 = time.perf_counter()
-            oracle.decode_mask(Ip, Iz, layer.rows, layer.cols)
+            M_ref = oracle.decode_mask(Ip, Iz, layer.rows, layer.cols)
             sec = time.perf_counter() - t0
             cpu = {"value": work_bytes / sec / 1e9, "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle",
                    "sample": "the whole index decode, once", "seconds": sec}
+            bad = int((wl["out"].cpu().numpy().view(np.uint32) != synth.pack_mask(M_ref)).sum())
+            parity = {"mask_words_differing": bad, "against": "oracle"}
+            if bad:
+                raise SystemExit("the timed kernel's mask disagrees with the oracle in %d words" % bad)
         else:
-            flops, sec, text, _ = oracle_sample_run(layer, batch, 15.0)
+            flops, sec, text, rows_sample, y_ref = oracle_sample_run(layer, batch, 15.0)
             cpu = {"value": flops / sec / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
                    "sample": text, "seconds": sec}
+            # the rows the oracle has just computed, against what the timed kernel left in Y
+            y_gpu = Y[:rows_sample].float().cpu().numpy().astype(np.float64)
+            rel = float(np.linalg.norm(y_gpu - y_ref) / max(np.linalg.norm(y_ref), 1e-300))
+            parity = {"rel_fro": rel, "rows": int(rows_sample), "tolerance": 5e-3, "against": "oracle (fp64)"}
+            if not rel <= 5e-3:
+                raise SystemExit("the timed kernel's Y disagrees with the oracle: relative Frobenius error %g" % rel)
+
+    # ---- the other configurations (rank 0, after the headline numbers are taken)
+    others = []
+    if args.others and world == 1:
+        del wl, step
+        if not decode_only:
+            del Y
+        torch.cuda.empty_cache()
+        flush2 = torch.zeros(256 * 1024 * 1024 // 4, dtype=torch.int32, device="cuda")
+        for name, ob in OTHER_WORKLOADS:
+            if name == args.workload and (ob == batch or not ob):
+                continue
+            ow = setup_workload(B, name, ob)
+            l0 = B.launch_count()
+            ts = time_calls(ow["step"], args.other_steps, 3, flush2)
+            nl = (B.launch_count() - l0) / (args.other_steps + 3)
+            ms = float(np.mean(ts))
+            others.append({"workload": name, "batch": ow["batch"], "kernel": kernel_label(B, ow["layer"], ow["batch"]),
+                           "ms": ms, "ms_median": float(np.median(ts)), "launches_per_step": nl,
+                           "algorithmic_bytes": ow["work_bytes"], "dense_flops": ow["work_flops"],
+                           "roofline": roofline_of(name, ow["batch"], ow["work_bytes"], ow["work_flops"], ms, peaks)})
+            del ow
+        if B.device_status() != 0:
+            raise SystemExit("device status word is not clean after the other workloads: %d" % B.device_status())
 
     line = {
         "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
@@ -362,7 +428,7 @@ def run_ours(args):
         "dtype": "u32" if decode_only else "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "batch": batch, "rows": layer.rows, "cols": layer.cols,
                    "tile": [layer.tile_rows, layer.tile_cols], "rank": layer.rank, "density": layer.density,
-                   "kernel": "decode" if decode_only else B.ALGO_NAMES[B.masked_gemm_choice(layer, batch)],
+                   "kernel": kernel_label(B, layer, batch),
                    "l2": "inputs larger than L2" if flush is None else "L2 flushed between timed calls (256 MiB rewrite)",
                    "algorithmic_bytes": work_bytes, "dense_flops": work_flops,
                    "effective_hbm_gbs": work_bytes / (ms_per_step * 1e-3) / 1e9},
@@ -372,6 +438,10 @@ def run_ours(args):
         line["e2e"] = e2e
     if cpu:
         line["cpu_baseline"] = cpu
+    if parity:
+        line["parity"] = parity
+    if others:
+        line["others"] = others
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -387,6 +457,9 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the batch of the workload")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", dest="others", action="store_false",
+                    help="skip the other configurations (reported in the \"others\" array of the line)")
+    ap.add_argument("--other-steps", type=int, default=30)
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 50 and args.warmup == 5:

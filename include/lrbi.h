@@ -30,6 +30,25 @@
  * detected on the host before anything is launched and reported by the return code; no
  * call aborts, throws or traps.  There is no CPU fallback: without a usable sm_100 device
  * a compute call returns LRBI_ERR_CUDA.
+ *
+ * Timeouts.  Every wait inside a kernel is bounded (about two seconds); a wait that runs out
+ * leaves a code in a per-device status word, the kernel ends early and its output is
+ * incomplete.  The asynchronous calls (lrbi_decode_mask, lrbi_masked_gemm, ..._static) cannot
+ * know this when they return.  The contract is: a call that synchronises
+ * (lrbi_layer_forward_host, lrbi_device_status, lrbi_last_device_error) reads the word; once
+ * it has been seen non-zero, every compute call on that device returns LRBI_ERR_TIMEOUT and
+ * launches nothing until lrbi_device_status(1) clears it.  A caller of the asynchronous calls
+ * checks lrbi_device_status after synchronising its stream.
+ *
+ * Threads.  Entry points may be called from several host threads; the library's own lazily
+ * built state is guarded by one lock.  Two calls that use the K-split buffer of
+ * lrbi_masked_gemm (or the fixed array of lrbi_masked_gemm_static) at the same time on
+ * different streams race on the device: order them.
+ *
+ * Non-finite values.  A NaN/Inf stored in a PRUNED weight never reaches Y (the weight is
+ * selected away).  Activations must be finite: the tensor-core kernels zero the pruned weight
+ * and still multiply, so an Inf/NaN in X at a pruned column gives NaN there, while the
+ * CUDA-core kernels skip the product; which kernel runs depends on the batch.
  */
 #ifndef LRBI_H_
 #define LRBI_H_
@@ -52,7 +71,8 @@ typedef enum {
     LRBI_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer          */
     LRBI_ERR_UNSUPPORTED = 2, /* a shape, dtype or kernel choice this library does not cover   */
     LRBI_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed (see lrbi_last_cuda_error)  */
-    LRBI_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up (see lrbi_device_status)   */
+    LRBI_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up earlier on this device and has
+                                 been seen by a synchronising call; cleared by lrbi_device_status(1) */
     LRBI_ERR_TOO_LARGE = 5    /* the problem needs more fixed scratch than the library carries   */
 } lrbi_status;
 
@@ -101,8 +121,9 @@ LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t 
 /*
  * Fused decode + prune + dense product (Eq. 3; masking layer of Sections 2 and 2.2):
  *       Y[b][o] = sum_i  Ia[o][i] ? X[b][i] * W[o][i] : 0      (fp32 accumulation)
- * The decoded index never reaches device memory.  A pruned weight is selected away, not
- * multiplied by zero, so a NaN/Inf stored in a pruned position does not reach Y.
+ * The decoded index never reaches device memory.  A pruned weight is selected away (its bf16
+ * pattern is replaced by +0 or its product is skipped), so a NaN/Inf stored in a pruned
+ * position does not reach Y.  X must be finite (see "Non-finite values" above).
  *   W      device, bf16 bit patterns, [rows][cols] row-major
  *   X      device, bf16 bit patterns, [batch][cols] row-major
  *   Y      device, [batch][rows] row-major, bf16 (round to nearest even) or fp32 per y_dtype
@@ -171,14 +192,42 @@ LRBI_API lrbi_status lrbi_layer_destroy(lrbi_layer *layer);
 /* Which kernel LRBI_ALGO_AUTO would run for this layout and batch (an LRBI_ALGO_* value). */
 LRBI_API int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batch);
 
+/*
+ * How lrbi_masked_gemm would run a call on the current device (nothing is launched).  For
+ * LRBI_ALGO_TENSOR the fields say which instantiation of the tcgen05 kernel runs; for the other
+ * kernels only `algo` is meaningful (k_splits = 1, the rest 0).
+ */
+typedef struct {
+    int32_t algo;          /* the LRBI_ALGO_* value that runs (LRBI_ALGO_AUTO resolved)             */
+    int32_t batch_tile;    /* batch rows per output tile                                            */
+    int32_t cta_pair;      /* 1: two CTAs of a cluster share a 256-row tile (tcgen05 cta_group::2)  */
+    int32_t panel_columns; /* columns of the index decoded per step inside the kernel (256 or 64)   */
+    int32_t k_splits;      /* thread blocks along the reduction; > 1 means fp32 partial sums + a second kernel */
+    int32_t stages;        /* operand stages in shared memory                                       */
+    uint64_t scratch_bytes;/* bytes of partial sums (what lrbi_masked_gemm_static_bytes reports)    */
+} lrbi_gemm_plan;
+LRBI_API lrbi_status lrbi_masked_gemm_plan(const lrbi_layout *layout, int32_t batch, int32_t algo,
+                                           lrbi_gemm_plan *plan);
+
 /* Kernels launched by this library since it was loaded (all entry points, this process). */
 LRBI_API uint64_t lrbi_launch_count(void);
 
 /*
  * Device-side status word of the current device: 0, or a code left by a kernel whose bounded
- * wait (pipeline barrier) ran out.  Synchronises the device.  `clear` != 0 resets it.
+ * wait (pipeline barrier) ran out.  Synchronises the device.  `clear` != 0 resets it and
+ * lifts the LRBI_ERR_TIMEOUT refusal of later calls.  Returns -1 if a CUDA call failed.
  */
 LRBI_API int32_t lrbi_device_status(int32_t clear);
+LRBI_API int32_t lrbi_last_device_error(void); /* lrbi_device_status(0) */
+
+/*
+ * Self-test of the timeout path (no counterpart in the paper).  Launches one tiny kernel whose single
+ * thread waits, with the same bounded wait the pipeline kernels use but a limit of `limit_us`
+ * microseconds (at most 100 000), on a barrier that nothing signals.  The wait gives up, the kernel
+ * returns normally and the status word of the device then holds 0x600.  Nothing hangs or traps; it is
+ * how the tests show that a timeout is recorded, reported (LRBI_ERR_TIMEOUT) and cleared.
+ */
+LRBI_API lrbi_status lrbi_selftest_bounded_wait(uint32_t limit_us, void *stream);
 
 LRBI_API const char *lrbi_status_string(lrbi_status s);
 LRBI_API int32_t lrbi_last_cuda_error(void); /* cudaError_t / CUresult of the last failed call, else 0 */

@@ -31,6 +31,13 @@ class LrbiError(RuntimeError):
         super().__init__("%s: %s (status %d, cuda error %d)" % (what, status_string(code), code, lib().lrbi_last_cuda_error()))
 
 
+class GemmPlan(ctypes.Structure):
+    """lrbi_gemm_plan: how lrbi_masked_gemm would run a call."""
+    _fields_ = [("algo", ctypes.c_int32), ("batch_tile", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
+                ("panel_columns", ctypes.c_int32), ("k_splits", ctypes.c_int32), ("stages", ctypes.c_int32),
+                ("scratch_bytes", ctypes.c_uint64)]
+
+
 class Layout(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int32), ("cols", ctypes.c_int32), ("tile_rows", ctypes.c_int32),
                 ("tile_cols", ctypes.c_int32), ("rank", ctypes.c_int32)]
@@ -75,6 +82,12 @@ def lib():
         L.lrbi_layer_destroy.restype = i32
         L.lrbi_masked_gemm_choice.argtypes = [lp, i32]
         L.lrbi_masked_gemm_choice.restype = i32
+        L.lrbi_masked_gemm_plan.argtypes = [lp, i32, i32, ctypes.POINTER(GemmPlan)]
+        L.lrbi_masked_gemm_plan.restype = i32
+        L.lrbi_last_device_error.argtypes = []
+        L.lrbi_last_device_error.restype = i32
+        L.lrbi_selftest_bounded_wait.argtypes = [ctypes.c_uint32, vp]
+        L.lrbi_selftest_bounded_wait.restype = i32
         L.lrbi_launch_count.argtypes = []
         L.lrbi_launch_count.restype = ctypes.c_uint64
         L.lrbi_device_status.argtypes = [i32]
@@ -102,6 +115,23 @@ def device_status(clear: bool = False) -> int:
 def masked_gemm_choice(layer, batch: int) -> int:
     lay = Layout.of(layer)
     return int(lib().lrbi_masked_gemm_choice(ctypes.byref(lay), batch))
+
+
+def masked_gemm_plan(layer, batch: int, algo: int = ALGO_AUTO) -> GemmPlan:
+    """The kernel instantiation lrbi_masked_gemm would run (nothing is launched)."""
+    lay = Layout.of(layer)
+    plan = GemmPlan()
+    rc = lib().lrbi_masked_gemm_plan(ctypes.byref(lay), batch, algo, ctypes.byref(plan))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_masked_gemm_plan")
+    return plan
+
+
+def selftest_bounded_wait(limit_us: int = 1000, stream=None) -> None:
+    """Runs the kernel whose bounded wait is meant to give up (leaves 0x600 in the status word)."""
+    rc = lib().lrbi_selftest_bounded_wait(limit_us, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_selftest_bounded_wait")
 
 
 def _stream_ptr(stream):
@@ -183,9 +213,12 @@ def lrbi_masked_gemm_static(layer, W: torch.Tensor, ip: torch.Tensor, iz: torch.
     keep them on one stream.
     """
     lay = Layout.of(layer)
-    batch = X.shape[0]
-    if tuple(W.shape) != (lay.rows, lay.cols) or X.dim() != 2 or X.shape[1] != lay.cols:
+    L = lib()
+    if X.dim() != 2 or tuple(W.shape) != (lay.rows, lay.cols) or X.shape[1] != lay.cols:
         raise ValueError("W / X shapes do not match the layout")
+    if ip.numel() != L.lrbi_packed_ip_words(ctypes.byref(lay)) or iz.numel() != L.lrbi_packed_iz_words(ctypes.byref(lay)):
+        raise ValueError("packed factor sizes do not match the layout")
+    batch = X.shape[0]
     if tuple(Y.shape) != (batch, lay.rows) or Y.dtype not in (torch.bfloat16, torch.float32):
         raise ValueError("Y must be [batch, rows] bf16 or fp32")
     code = Y_BF16 if Y.dtype == torch.bfloat16 else Y_F32

@@ -13,7 +13,10 @@ __device__ int g_device_status = 0;
 static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_last_cuda_error{0};
 static std::mutex g_mutex;
-static int *g_status_ptr[64] = {nullptr};
+static int *g_status_ptr[LRBI_MAX_DEVICES] = {nullptr};
+static std::atomic<int> g_timeout_seen[LRBI_MAX_DEVICES];   // sticky: set when a synchronising call reads a non-zero status word
+
+std::mutex &lib_mutex() { return g_mutex; }
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 void note_cuda_error(int code) { g_last_cuda_error.store(code, std::memory_order_relaxed); }
@@ -21,7 +24,7 @@ void note_cuda_error(int code) { g_last_cuda_error.store(code, std::memory_order
 int *device_status_ptr()
 {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= LRBI_MAX_DEVICES) return nullptr;
     std::lock_guard<std::mutex> lock(g_mutex);
     if (!g_status_ptr[dev]) {
         void *p = nullptr;
@@ -30,6 +33,35 @@ int *device_status_ptr()
         g_status_ptr[dev] = static_cast<int *>(p);
     }
     return g_status_ptr[dev];
+}
+
+bool device_timeout_seen()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= LRBI_MAX_DEVICES) return false;
+    return g_timeout_seen[dev].load(std::memory_order_relaxed) != 0;
+}
+
+// Reads the status word of the current device; the caller has synchronised whatever it cares about.
+// A non-zero word makes every later compute call on the device return LRBI_ERR_TIMEOUT until it is cleared.
+static int read_status_word(bool clear)
+{
+    int *p = device_status_ptr();
+    if (!p) return -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int v = 0;
+    cudaError_t e = cudaMemcpy(&v, p, sizeof v, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { note_cuda_error((int)e); return -1; }
+    if (v != 0) g_timeout_seen[dev].store(1, std::memory_order_relaxed);
+    if (clear) {
+        if (v != 0) {
+            const int zero = 0;
+            cudaMemcpy(p, &zero, sizeof zero, cudaMemcpyHostToDevice);
+        }
+        g_timeout_seen[dev].store(0, std::memory_order_relaxed);
+    }
+    return v;
 }
 
 static bool layout_ok(const lrbi_layout *l)
@@ -81,6 +113,7 @@ lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t *ip, cons
 {
     if (!layout_ok(layout) || !ip || !iz || !mask_out) return LRBI_ERR_INVALID_ARG;
     if (!aligned16(ip) || !aligned16(iz) || !aligned16(mask_out)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
     const Geo g = make_geo(*layout);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (algo) {
@@ -107,6 +140,7 @@ lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const
     if (!layout_ok(layout) || !W || !ip || !iz || !X || !Y || batch < 1) return LRBI_ERR_INVALID_ARG;
     if (y_dtype != LRBI_Y_BF16 && y_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
     if (!aligned16(W) || !aligned16(ip) || !aligned16(iz) || !aligned16(X) || !aligned16(Y)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
     const Geo g = make_geo(*layout);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (algo == LRBI_ALGO_AUTO) algo = choose_gemm(g, batch);
@@ -126,6 +160,7 @@ lrbi_status lrbi_masked_gemm_static(const lrbi_layout *layout, const uint16_t *W
     if (!layout_ok(layout) || !W || !ip || !iz || !X || !Y || batch < 1) return LRBI_ERR_INVALID_ARG;
     if (y_dtype != LRBI_Y_BF16 && y_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
     if (!aligned16(W) || !aligned16(ip) || !aligned16(iz) || !aligned16(X) || !aligned16(Y)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
     return launch_gemm_tc_static(make_geo(*layout), W, ip, iz, X, batch, Y, y_dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -140,17 +175,33 @@ uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_rela
 
 int32_t lrbi_device_status(int32_t clear)
 {
-    int *p = device_status_ptr();
-    if (!p) return -1;
-    int v = 0;
     cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemcpy(&v, p, sizeof v, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) { note_cuda_error((int)e); return -1; }
-    if (clear && v != 0) {
-        const int zero = 0;
-        cudaMemcpy(p, &zero, sizeof zero, cudaMemcpyHostToDevice);
+    return read_status_word(clear != 0);
+}
+
+int32_t lrbi_last_device_error(void) { return lrbi_device_status(0); }
+
+lrbi_status lrbi_selftest_bounded_wait(uint32_t limit_us, void *stream)
+{
+    return launch_bounded_wait_selftest(limit_us, static_cast<cudaStream_t>(stream));
+}
+
+lrbi_status lrbi_masked_gemm_plan(const lrbi_layout *layout, int32_t batch, int32_t algo, lrbi_gemm_plan *plan)
+{
+    if (!layout_ok(layout) || batch < 1 || !plan) return LRBI_ERR_INVALID_ARG;
+    const Geo g = make_geo(*layout);
+    if (algo == LRBI_ALGO_AUTO) algo = choose_gemm(g, batch);
+    std::memset(plan, 0, sizeof *plan);
+    plan->algo = algo;
+    plan->k_splits = 1;
+    switch (algo) {
+    case LRBI_ALGO_GENERIC: return LRBI_OK;
+    case LRBI_ALGO_GEMV: return gemv_supported(g, batch) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    case LRBI_ALGO_STREAM: return stream_mma_supported(g, batch) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    case LRBI_ALGO_TENSOR: return gemm_tc_plan(g, batch, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    default: return LRBI_ERR_INVALID_ARG;
     }
-    return v;
 }
 
 const char *lrbi_status_string(lrbi_status s)
@@ -269,6 +320,9 @@ lrbi_status lrbi_layer_forward_host(lrbi_layer *L, const uint16_t *X_host, int32
     cudaError_t e4 = cudaStreamSynchronize(L->s_out);
     if (e == cudaSuccess) e = e2 != cudaSuccess ? e2 : (e3 != cudaSuccess ? e3 : e4);
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
+    // every kernel of this call has finished: a bounded wait that gave up left its code in the status word,
+    // and Y_host is then incomplete
+    if (st == LRBI_OK && read_status_word(false) != 0) return LRBI_ERR_TIMEOUT;
     return st;
 }
 

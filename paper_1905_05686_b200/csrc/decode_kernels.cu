@@ -199,24 +199,6 @@ constexpr int WIDE_WORDS = 32;          // mask words (1024 columns = one 128-by
 constexpr int WIDE_PITCH = 36;          // words between planes in shared memory (16-byte aligned, spreads banks)
 constexpr int WIDE_MAX_RANK = 256;
 
-// 32 x 32 bit-matrix transpose across a warp: lane L gives x_L, lane l receives the word whose bit L is
-// bit l of x_L -- the 32 words that 32 __ballot_sync votes on ((x >> l) & 1) would give.
-__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane)
-{
-#pragma unroll
-    for (int stage = 0; stage < 5; ++stage) {
-        const int j = 16 >> stage;
-        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
-                         : stage == 3 ? 0x33333333u : 0x55555555u;
-        const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, j);
-        const bool upper = (lane & j) != 0;
-        const uint32_t sh = upper ? (y >> j) : (y << j);
-        const uint32_t keep = upper ? ~m : m;
-        x = (x & keep) | (sh & ~keep);
-    }
-    return x;
-}
-
 // SEGQ = 128-column quads per run of columns that lies inside one tile (8: the whole block).
 template <int SEGQ>
 __global__ void __launch_bounds__(DEC_THREADS, SEGQ <= 2 ? 8 : 4)

@@ -36,6 +36,8 @@
 // TMA thread drains (bounded) the copies it has in flight, and tensor memory is freed before exit.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "lrbi_common.cuh"
 
 namespace lrbi {
@@ -78,7 +80,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // `code` and raises the abort flag).  The limit is counted on the SM's own cycle counter, which is
 // cheap to read; it is looked at once every 64 unsuccessful tries.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
-                                          int *status, int code)
+                                          int *status, int code, long long limit = TC_WAIT_LIMIT_CYCLES)
 {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = 0;
@@ -93,7 +95,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if ((spins & 63u) == 0) {
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > TC_WAIT_LIMIT_CYCLES) {
+            else if (now - t0 > limit) {
                 atomicCAS(status, 0, code);
                 *abort_flag = 1;
                 __threadfence_block();
@@ -278,46 +280,6 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 // 8i + 7 - g, so that `word << g` leaves the four bits of group g on the sign positions of the
 // four bytes.  column_of_bit is the inverse (which column a ballot lane stands for).
 __device__ __forceinline__ int column_of_bit(int bit) { return 4 * (7 - (bit & 7)) + (bit >> 3); }
-
-// 32 x 32 bit-matrix transpose across a warp: lane L gives the word x_L, lane l receives the word
-// whose bit L is bit l of x_L.  Five butterfly stages of one shuffle each.  It yields the same
-// 32 words as 32 __ballot_sync votes on ((x >> l) & 1), l = 0..31, at a sixth of the instructions.
-__device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane)
-{
-#pragma unroll
-    for (int stage = 0; stage < 5; ++stage) {
-        const int j = 16 >> stage;
-        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
-                         : stage == 3 ? 0x33333333u : 0x55555555u;
-        const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, j);
-        const bool upper = (lane & j) != 0;
-        const uint32_t sh = upper ? (y >> j) : (y << j);
-        const uint32_t keep = upper ? ~m : m;
-        x = (x & keep) | (sh & ~keep);
-    }
-    return x;
-}
-
-// Four independent transposes with their shuffles interleaved (latency of one, work of four).
-__device__ __forceinline__ void transpose32_x4(uint32_t (&x)[4], int lane)
-{
-#pragma unroll
-    for (int stage = 0; stage < 5; ++stage) {
-        const int j = 16 >> stage;
-        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
-                         : stage == 3 ? 0x33333333u : 0x55555555u;
-        const bool upper = (lane & j) != 0;
-        const uint32_t keep = upper ? ~m : m;
-        uint32_t y[4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) y[t] = __shfl_xor_sync(0xFFFFFFFFu, x[t], j);
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            const uint32_t sh = upper ? (y[t] >> j) : (y[t] << j);
-            x[t] = (x[t] & keep) | (sh & ~keep);
-        }
-    }
-}
 
 // Zero the pruned halves of the eight bf16 values of one 16-byte chunk.  `bits` holds the index
 // bits of the row's 32 columns in the permuted order above; chunk j uses groups 2j and 2j+1.
@@ -521,7 +483,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                     z[t] = (pi < npairs && c0 + col < g.cols) ? iz_stage[col * g.kw + lb] : 0u;
                     if (lb == g.kw - 1) z[t] &= tail;
                 }
-                transpose32_x4(z, lane);
+                warp_transpose32_x4(z, lane);
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
                     const int pi = dw + TC_DECODE_WARPS * (n0 + t);
@@ -708,6 +670,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     }
 }
 
+// The give-up path of the pipeline's bounded wait, exercised on its own: one thread waits, with a short
+// limit, on a barrier that nothing arrives at.  The wait runs out, the code lands in the status word and
+// the kernel returns normally.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles, int *status)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(&bar, 0, &abort_flag, status, DEV_TIMEOUT_SELFTEST, limit_cycles);
+    }
+}
+
+lrbi_status launch_bounded_wait_selftest(unsigned limit_us, cudaStream_t s)
+{
+    int *status = device_status_ptr();
+    if (!status) return LRBI_ERR_CUDA;
+    if (limit_us > 100000u) limit_us = 100000u;          // a tenth of a second at most
+    bounded_wait_selftest_kernel<<<1, 32, 0, s>>>((long long)limit_us * 2000ll, status);   // about 2 cycles per ns
+    count_launch();
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
+    return LRBI_OK;
+}
+
 // Sum of the K-split partial results: Y[b][o] = sum_z partials[z][b][o].
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ partials, int splits, long long n, void *__restrict__ Y, int y_dtype)
@@ -730,6 +719,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 static EncodeTiledFn get_encode_fn()
 {
     static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> lock(lib_mutex());
     if (!fn) {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -751,19 +741,16 @@ bool gemm_tc_supported(const Geo &g, int batch)
     return true;
 }
 
-// Index words per panel row: 256-column panels when every panel then lies inside one tile.
-static int panel_words(const Geo &g) { return (g.gc == 1 || (g.tn % 256) == 0) ? 8 : 2; }
-
+// Library-owned buffer for K-split partial sums, one per device, grown on demand (under the library lock).
 struct Workspace {
     float *ptr = nullptr;
     size_t bytes = 0;
 };
-static Workspace g_ws[64];
+static Workspace g_ws[LRBI_MAX_DEVICES];
 
-static float *workspace(size_t bytes)
+static float *workspace(int dev, size_t bytes)
 {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(lib_mutex());
     Workspace &w = g_ws[dev];
     if (w.bytes < bytes) {
         if (w.ptr) cudaFree(w.ptr);
@@ -774,17 +761,44 @@ static float *workspace(size_t bytes)
     return w.ptr;
 }
 
-// How the reduction over K is cut: `splits` blocks along grid z, each `kb_per_split` K blocks long.
-struct SplitPlan { int splits, kb_per_split, row_blocks; };
-static SplitPlan plan_splits(const Geo &g, int batch, int bn, bool pair, int sm_count)
+// Everything the host decides about one launch of the tensor-core kernel: which instantiation runs, how
+// the reduction over K is cut, how many operand stages fit.  One function, so that the launcher, the
+// scratch-size query and the plan query of the C ABI cannot disagree.
+struct TcPlan {
+    int bn;              // batch columns per output tile
+    int pw;              // index words per panel row (8: 256-column panels, 2: 64-column panels)
+    bool pair;           // CTA pairs (cta_group::2)
+    int row_blocks;      // 128-row blocks along grid y (pair mode: an even number, two per cluster)
+    int splits;          // blocks along the reduction (grid z)
+    int kb_per_split;    // K blocks per split (a multiple of 4: splits start on panel boundaries)
+    int stages;          // operand stages in shared memory
+    size_t smem;         // dynamic shared memory per block
+    size_t scratch;      // bytes of fp32 partial sums (0 when K is not split)
+};
+
+static bool use_pairs(const Geo &g, int batch, int sm_count)
 {
-    SplitPlan p;
+    if (batch <= 128) return false;
+    const long long pair_blocks = 2LL * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) * ((batch + 255) / 256);
+    return pair_blocks * 2 >= 3LL * sm_count;
+}
+
+static bool make_tc_plan(const Geo &g, int batch, int sm_count, TcPlan *out)
+{
+    if (!gemm_tc_supported(g, batch)) return false;
+    TcPlan p;
+    // large batch: CTA pairs share each X tile, unless there are too few pairs of tiles to fill the chip
+    // (a layer with few rows): then single CTAs with 128-row batch tiles give twice as many blocks
+    p.pair = use_pairs(g, batch, sm_count);
+    p.bn = batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : (batch <= 128 || !p.pair) ? 128 : 256;
+    // index words per panel row: 256-column panels when every panel then lies inside one tile
+    p.pw = (g.gc == 1 || (g.tn % 256) == 0) ? 8 : 2;
     const int nkb = (g.cols + TC_BK - 1) / TC_BK;
-    p.row_blocks = pair ? 2 * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) : (g.rows + TC_BM - 1) / TC_BM;
-    const int tiles = ((batch + bn - 1) / bn) * p.row_blocks;
+    p.row_blocks = p.pair ? 2 * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) : (g.rows + TC_BM - 1) / TC_BM;
+    const int tiles = ((batch + p.bn - 1) / p.bn) * p.row_blocks;
     // split K when the output tiles alone cannot occupy the chip (small batch: bandwidth-bound)
     int splits = 1;
-    if (batch <= bn && tiles < 2 * sm_count) {        // one batch tile: the small-batch, bandwidth-bound case
+    if (batch <= p.bn && tiles < 2 * sm_count) {      // one batch tile: the small-batch, bandwidth-bound case
         splits = (2 * sm_count + tiles - 1) / tiles;
         splits = splits > nkb / 4 ? (nkb / 4 > 0 ? nkb / 4 : 1) : splits;   // at least 4 K blocks per split
         if (splits > 32) splits = 32;
@@ -793,13 +807,41 @@ static SplitPlan plan_splits(const Geo &g, int batch, int bn, bool pair, int sm_
     kb_per_split = (kb_per_split + 3) / 4 * 4;                               // splits start on panel boundaries
     p.splits = (nkb + kb_per_split - 1) / kb_per_split;                      // no empty split
     p.kb_per_split = kb_per_split;
-    return p;
+    p.scratch = p.splits > 1 ? (size_t)p.splits * batch * g.rows * sizeof(float) : 0;
+
+    // As many stages as let two blocks share an SM (at least three); if two cannot fit (large ranks need
+    // more room for planes and factor staging), one block with up to six stages.  Two resident blocks
+    // overlap one's epilogue and hand-overs with the other's MMAs and double the copies in flight.
+    // (an SM has 228 KB of shared memory; each resident block also reserves 1 KB)
+    const size_t b_stage = (size_t)(p.pair ? p.bn / 2 : p.bn) * TC_BK * 2;
+    const size_t extras = (size_t)(2 * TC_BM * p.pw + g.kw * 32 * (p.pw == 8 ? 12 : p.pw) + p.pw * 32 * g.kw + TC_BM * g.kw) * 4 + sizeof(TcCtl);
+    const size_t per_stage = TC_A_STAGE_BYTES + b_stage;
+    const size_t half_sm = 113 * 1024, whole_sm = 224 * 1024;
+    int stages = (int)((half_sm - extras) / per_stage);
+    if (extras > half_sm || stages < 3) stages = (int)((whole_sm - extras) / per_stage);
+    if (stages > 6) stages = 6;
+    if (stages < 2) return false;
+    p.stages = stages;
+    p.smem = (size_t)stages * per_stage + extras;
+    const unsigned nbt = (unsigned)((batch + p.bn - 1) / p.bn);
+    if ((p.pair ? p.row_blocks / 2 : p.row_blocks) > 65535 || p.splits > 65535 || nbt > 0x3FFFFFFFu) return false;
+    *out = p;
+    return true;
+}
+
+static int device_sm_count(int *dev_out)
+{
+    int dev = 0, sm_count = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= LRBI_MAX_DEVICES) { *dev_out = -1; return sm_count; }
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    *dev_out = dev;
+    return sm_count;
 }
 
 template <int BN, int PW, bool PAIR>
-static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                             const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count,
-                             float *fixed_scratch = nullptr, size_t fixed_bytes = 0)
+static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const uint16_t *W, const uint32_t *ip,
+                             const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype,
+                             cudaStream_t s, float *partials)
 {
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) { note_cuda_error(-1); return LRBI_ERR_CUDA; }
@@ -820,50 +862,23 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
-    constexpr int B_STAGE = (PAIR ? BN / 2 : BN) * TC_BK * 2;
-    const SplitPlan plan = plan_splits(g, batch, BN, PAIR, sm_count);
-    const int row_blocks = plan.row_blocks, splits = plan.splits, kb_per_split = plan.kb_per_split;
-
-    // Pair mode: three stages when two blocks then fit one SM (k <= 64); larger ranks need more room for
-    // planes and factor staging, run one block per SM and get six stages.
-    const size_t extras = (size_t)(2 * TC_BM * PW + g.kw * 32 * (PW == 8 ? 12 : PW) + PW * 32 * g.kw + TC_BM * g.kw) * 4 + sizeof(TcCtl);
-    const size_t per_stage = TC_A_STAGE_BYTES + B_STAGE;
-    // As many stages as let two blocks share an SM (at least three); if two cannot fit, one block with
-    // up to six stages.  Two resident blocks overlap one's epilogue and hand-overs with the other's MMAs
-    // and double the copies in flight.
-    // (an SM has 228 KB of shared memory; each resident block also reserves 1 KB)
-    const size_t half_sm = 113 * 1024, whole_sm = 224 * 1024;
-    int stages = (int)((half_sm - extras) / per_stage);
-    if (extras > half_sm || stages < 3) stages = (int)((whole_sm - extras) / per_stage);
-    if (stages > 6) stages = 6;
-    if (stages < 2) return LRBI_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)stages * per_stage + extras;
-
-    float *partials = nullptr;
-    if (splits > 1) {
-        const size_t need = (size_t)splits * batch * g.rows * sizeof(float);
-        if (fixed_scratch) {                             // caller forbids allocation: fixed array or nothing
-            if (need > fixed_bytes) return LRBI_ERR_TOO_LARGE;
-            partials = fixed_scratch;
-        } else {
-            partials = workspace(need);
-            if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
+    auto kern = gemm_tc_kernel<BN, PW, PAIR>;
+    {
+        // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the function
+        static bool attr_done[LRBI_MAX_DEVICES] = {false};
+        std::lock_guard<std::mutex> lock(lib_mutex());
+        if (!attr_done[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
+            if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
+            attr_done[dev] = true;
         }
     }
-    auto kern = gemm_tc_kernel<BN, PW, PAIR>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
-        if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
-        attr_done = true;
-    }
     const unsigned nbt = (unsigned)((batch + BN - 1) / BN);
-    dim3 grid(PAIR ? 2 * nbt : nbt, (unsigned)(PAIR ? row_blocks / 2 : row_blocks), (unsigned)splits);
-    if (grid.y > 65535 || grid.z > 65535) return LRBI_ERR_UNSUPPORTED;
+    dim3 grid(PAIR ? 2 * nbt : nbt, (unsigned)(PAIR ? plan.row_blocks / 2 : plan.row_blocks), (unsigned)plan.splits);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(TC_THREADS);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;      // the pair must lie along x: other shapes are refused
@@ -873,13 +888,13 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int *status = device_status_ptr();
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, ip, iz, batch, Y, y_dtype, partials, kb_per_split, stages, status);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, ip, iz, batch, Y, y_dtype, partials, plan.kb_per_split, plan.stages, status);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
-    if (splits > 1) {
+    if (plan.splits > 1) {
         const long long n = (long long)batch * g.rows;
-        splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, splits, n, Y, y_dtype);
+        splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, plan.splits, n, Y, y_dtype);
         count_launch();
         e = cudaGetLastError();
         if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
@@ -887,40 +902,55 @@ static lrbi_status launch_tc(const Geo &g, const uint16_t *W, const uint32_t *ip
     return LRBI_OK;
 }
 
-template <int BN>
-static lrbi_status launch_tc_kw(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                                const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int sm_count,
-                                float *fixed_scratch = nullptr, size_t fixed_bytes = 0)
+// `fixed_scratch` != nullptr: the caller forbids allocation, partial sums go there (fixed_bytes) or nowhere.
+static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
+                          const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s,
+                          float *fixed_scratch, size_t fixed_bytes)
 {
-    return panel_words(g) == 8 ? launch_tc<BN, 8, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, fixed_scratch, fixed_bytes)
-                               : launch_tc<BN, 2, false>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, fixed_scratch, fixed_bytes);
-}
-
-static bool use_pairs(const Geo &g, int batch, int sm_count)
-{
-    if (batch <= 128) return false;
-    const long long pair_blocks = 2LL * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) * ((batch + 255) / 256);
-    return pair_blocks * 2 >= 3LL * sm_count;
+    if (!gemm_tc_supported(g, batch)) return LRBI_ERR_UNSUPPORTED;    // shape errors come before device errors
+    int dev = -1;
+    const int sm_count = device_sm_count(&dev);
+    if (dev < 0) return LRBI_ERR_CUDA;
+    TcPlan plan;
+    if (!make_tc_plan(g, batch, sm_count, &plan)) return LRBI_ERR_UNSUPPORTED;
+    if (fixed_scratch && plan.scratch > fixed_bytes) return LRBI_ERR_TOO_LARGE;   // before any launch
+    if (!device_status_ptr()) return LRBI_ERR_CUDA;
+    float *partials = nullptr;
+    if (plan.scratch) {
+        partials = fixed_scratch ? fixed_scratch : workspace(dev, plan.scratch);
+        if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
+    }
+#define LRBI_TC_CASE(BN_, PW_, PAIR_) \
+    if (plan.bn == BN_ && plan.pw == PW_ && plan.pair == PAIR_) \
+        return launch_tc<BN_, PW_, PAIR_>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials);
+    LRBI_TC_CASE(16, 8, false) LRBI_TC_CASE(16, 2, false)
+    LRBI_TC_CASE(32, 8, false) LRBI_TC_CASE(32, 2, false)
+    LRBI_TC_CASE(64, 8, false) LRBI_TC_CASE(64, 2, false)
+    LRBI_TC_CASE(128, 8, false) LRBI_TC_CASE(128, 2, false)
+    LRBI_TC_CASE(256, 8, true) LRBI_TC_CASE(256, 2, true)
+#undef LRBI_TC_CASE
+    return LRBI_ERR_UNSUPPORTED;
 }
 
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                            const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s)
 {
-    if (!gemm_tc_supported(g, batch)) return LRBI_ERR_UNSUPPORTED;
-    if (!device_status_ptr()) return LRBI_ERR_CUDA;
-    int dev = 0, sm_count = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (batch <= 16) return launch_tc_kw<16>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    if (batch <= 32) return launch_tc_kw<32>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    if (batch <= 64) return launch_tc_kw<64>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    if (batch <= 128) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    // large batch: CTA pairs share each X tile, unless there are too few pairs of tiles to fill the chip
-    // (a layer with few rows): then single CTAs with 128-row batch tiles give twice as many blocks
-    if (use_pairs(g, batch, sm_count))
-        return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count)
-                                   : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
-    return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count);
+    return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, nullptr, 0);
+}
+
+bool gemm_tc_plan(const Geo &g, int batch, lrbi_gemm_plan *out)
+{
+    int dev = -1;
+    const int sm_count = device_sm_count(&dev);
+    TcPlan p;
+    if (!make_tc_plan(g, batch, sm_count, &p)) return false;
+    out->batch_tile = p.bn;
+    out->cta_pair = p.pair ? 1 : 0;
+    out->panel_columns = p.pw * 32;
+    out->k_splits = p.splits;
+    out->stages = p.stages;
+    out->scratch_bytes = (uint64_t)p.scratch;
+    return true;
 }
 
 // --------------------------------------------------------------------------------------
@@ -930,12 +960,13 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
 // process ends.  In host code this name is only a handle for the runtime, never a device address;
 // the address a kernel may use comes from cudaGetSymbolAddress, asked once per device.
 static __device__ __align__(256) float g_static_scratch[LRBI_STATIC_SCRATCH_BYTES / sizeof(float)];
-static float *g_static_scratch_ptr[64] = {nullptr};
+static float *g_static_scratch_ptr[LRBI_MAX_DEVICES] = {nullptr};
 
 static float *static_scratch_ptr()
 {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= LRBI_MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(lib_mutex());
     if (!g_static_scratch_ptr[dev]) {                    // first call on this device (it is the current one)
         void *p = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
@@ -945,16 +976,12 @@ static float *static_scratch_ptr()
     return g_static_scratch_ptr[dev];
 }
 
-static int batch_tile(int batch) { return batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : batch <= 128 ? 128 : 256; }
-
 size_t gemm_tc_scratch_bytes(const Geo &g, int batch)
 {
-    int dev = 0, sm_count = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    const bool pair = use_pairs(g, batch, sm_count);
-    const SplitPlan p = plan_splits(g, batch, (batch > 128 && !pair) ? 128 : batch_tile(batch), pair, sm_count);
-    return p.splits > 1 ? (size_t)p.splits * batch * g.rows * sizeof(float) : 0;
+    int dev = -1;
+    const int sm_count = device_sm_count(&dev);
+    TcPlan p;
+    return make_tc_plan(g, batch, sm_count, &p) ? p.scratch : 0;
 }
 
 lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
@@ -962,19 +989,9 @@ lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_
 {
     if (!gemm_tc_supported(g, batch)) return LRBI_ERR_UNSUPPORTED;
     if (gemm_tc_scratch_bytes(g, batch) > LRBI_STATIC_SCRATCH_BYTES) return LRBI_ERR_TOO_LARGE;   // before any launch
-    if (!device_status_ptr()) return LRBI_ERR_CUDA;
     float *scratch = static_scratch_ptr();
     if (!scratch) return LRBI_ERR_CUDA;
-    int dev = 0, sm_count = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    const size_t cap = LRBI_STATIC_SCRATCH_BYTES;
-    if (batch <= 16) return launch_tc_kw<16>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
-    if (batch <= 32) return launch_tc_kw<32>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
-    if (batch <= 64) return launch_tc_kw<64>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
-    if (batch <= 128 || !use_pairs(g, batch, sm_count)) return launch_tc_kw<128>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
-    return panel_words(g) == 8 ? launch_tc<256, 8, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap)
-                               : launch_tc<256, 2, true>(g, W, ip, iz, X, batch, Y, y_dtype, s, sm_count, scratch, cap);
+    return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, scratch, LRBI_STATIC_SCRATCH_BYTES);
 }
 
 }  // namespace lrbi

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "lrbi.h"
 
 namespace lrbi {
@@ -34,11 +36,19 @@ enum : int {
     DEV_TIMEOUT_EMPTY = 0x200,  // a producer waited for a free stage
     DEV_TIMEOUT_ACCUM = 0x300,  // epilogue waited for the accumulator
     DEV_TIMEOUT_DRAIN = 0x400,  // drain of in-flight bulk copies on the abort path
-    DEV_BAD_SMEM_ALIGN = 0x500  // dynamic shared memory did not start on a 1024-byte boundary
+    DEV_BAD_SMEM_ALIGN = 0x500, // dynamic shared memory did not start on a 1024-byte boundary
+    DEV_TIMEOUT_SELFTEST = 0x600 // the self-test's wait on a barrier nobody signals (expected to run out)
 };
+
+constexpr int LRBI_MAX_DEVICES = 64;       // size of the per-device tables
+
+// One lock for the library's lazily initialised host state (per-device tables, the driver entry point,
+// the K-split buffer, function attributes).  Entry points may be called from several host threads.
+std::mutex &lib_mutex();
 
 // Device status word (one per device that loads the module) and the host-side accessors.
 int *device_status_ptr();                  // device address, resolved once per device
+bool device_timeout_seen();                // a synchronising call has seen a non-zero status word on the current device
 void count_launch(int n = 1);
 void note_cuda_error(int code);
 
@@ -59,6 +69,48 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
     return (uint16_t)(u >> 16);
 }
 
+#ifdef __CUDACC__
+// 32 x 32 bit-matrix transpose across a warp: lane L gives the word x_L, lane l receives the word
+// whose bit L is bit l of x_L.  Five butterfly stages of one shuffle each.  It yields the same
+// 32 words as 32 __ballot_sync votes on ((x >> l) & 1), l = 0..31, at a sixth of the instructions.
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane)
+{
+#pragma unroll
+    for (int stage = 0; stage < 5; ++stage) {
+        const int j = 16 >> stage;
+        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
+                         : stage == 3 ? 0x33333333u : 0x55555555u;
+        const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, j);
+        const bool upper = (lane & j) != 0;
+        const uint32_t sh = upper ? (y >> j) : (y << j);
+        const uint32_t keep = upper ? ~m : m;
+        x = (x & keep) | (sh & ~keep);
+    }
+    return x;
+}
+
+// Four independent transposes with their shuffles interleaved (latency of one, work of four).
+__device__ __forceinline__ void warp_transpose32_x4(uint32_t (&x)[4], int lane)
+{
+#pragma unroll
+    for (int stage = 0; stage < 5; ++stage) {
+        const int j = 16 >> stage;
+        const uint32_t m = stage == 0 ? 0x0000FFFFu : stage == 1 ? 0x00FF00FFu : stage == 2 ? 0x0F0F0F0Fu
+                         : stage == 3 ? 0x33333333u : 0x55555555u;
+        const bool upper = (lane & j) != 0;
+        const uint32_t keep = upper ? ~m : m;
+        uint32_t y[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) y[t] = __shfl_xor_sync(0xFFFFFFFFu, x[t], j);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const uint32_t sh = upper ? (y[t] >> j) : (y[t] << j);
+            x[t] = (x[t] & keep) | (sh & ~keep);
+        }
+    }
+}
+#endif
+
 // Kernel launchers (one translation unit each).
 lrbi_status launch_decode_ballot(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
 lrbi_status launch_decode_planes(const Geo &g, const uint32_t *ip, const uint32_t *iz, uint32_t *mask, cudaStream_t s);
@@ -74,7 +126,7 @@ bool stream_mma_supported(const Geo &g, int batch);
 lrbi_status launch_stream_mma(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                               const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 bool gemm_tc_supported(const Geo &g, int batch);
-// `partials` == nullptr lets the launcher use the library-owned buffer when it splits K.
+// When it splits K the launcher keeps fp32 partial sums in the library-owned buffer of the device.
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                            const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 
@@ -82,5 +134,7 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
 lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                                   const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 size_t gemm_tc_scratch_bytes(const Geo &g, int batch);   // fp32 partial sums the tensor-core path would keep
+lrbi_status launch_bounded_wait_selftest(unsigned limit_us, cudaStream_t s);
+bool gemm_tc_plan(const Geo &g, int batch, lrbi_gemm_plan *out);   // fills the tensor-core fields of the plan
 
 }  // namespace lrbi

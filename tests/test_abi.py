@@ -25,7 +25,7 @@ def declared_symbols():
 
 def test_every_declared_symbol_is_exported(lib):
     names = declared_symbols()
-    assert len(names) >= 13 and "lrbi_decode_mask" in names and "lrbi_masked_gemm" in names
+    assert len(names) >= 17 and "lrbi_decode_mask" in names and "lrbi_masked_gemm" in names
     L = ctypes.CDLL(lib.LIB_PATH)
     for n in names:
         assert hasattr(L, n), n
@@ -72,3 +72,20 @@ def test_kernel_choice_per_config(lib):
     assert lib.masked_gemm_choice(c, 16) == lib.ALGO_TENSOR
     assert lib.masked_gemm_choice(synth.CONFIGS["ffn_16384x4096"], 4096) == lib.ALGO_TENSOR
     assert lib.masked_gemm_choice(synth.Layer("odd", 37, 45, 16, 20, 7, 0.2), 5) == lib.ALGO_GENERIC
+
+
+def test_plan_query_runs_without_a_device(lib):
+    """The plan is host arithmetic: which instantiation of the tensor-core kernel a call would run."""
+    from paper_1905_05686_b200 import synth
+    p = lib.masked_gemm_plan(synth.CONFIGS["ffn_16384x4096"], 4096)
+    assert (p.algo, p.cta_pair, p.batch_tile, p.panel_columns, p.k_splits) == (lib.ALGO_TENSOR, 1, 256, 256, 1)
+    assert p.scratch_bytes == 0 and p.stages >= 3
+    p = lib.masked_gemm_plan(synth.CONFIGS["alexnet_fc"], 16)
+    assert p.algo == lib.ALGO_TENSOR and p.cta_pair == 0 and p.k_splits > 1
+    assert p.scratch_bytes == p.k_splits * 16 * 4096 * 4
+    assert lib.masked_gemm_static_bytes(synth.CONFIGS["alexnet_fc"], 16) == p.scratch_bytes
+    p = lib.masked_gemm_plan(synth.CONFIGS["alexnet_fc"], 1)
+    assert p.algo == lib.ALGO_GEMV and p.k_splits == 1
+    with pytest.raises(lib.LrbiError) as e:
+        lib.masked_gemm_plan(synth.Layer("odd", 37, 45, 16, 20, 7, 0.2), 64, lib.ALGO_TENSOR)
+    assert e.value.code == lib.ERR_UNSUPPORTED

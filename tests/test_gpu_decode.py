@@ -135,10 +135,10 @@ def test_degenerate_factors(algo):
         check(L, _algo(algo), p=p)                              # empty and full masks
 
 
-@pytest.mark.parametrize("algo", ["ballot", "planes"])
+@pytest.mark.parametrize("algo", ["ballot", "planes", "wide"])
 def test_bits_beyond_rank_are_ignored(algo):
     b = _b()
-    L = synth.Layer("pad", 64, 96, 32, 32, 5, 0.3)
+    L = synth.Layer("pad", 64, 96, 32, 32, 5, 0.3) if algo != "wide" else synth.Layer("pad", 64, 384, 32, 128, 5, 0.3)
     Ip, Iz = synth.make_factors(L)
     M = oracle.decode_mask(Ip, Iz, L.rows, L.cols)
     ipw = synth.pack_ip(Ip) | np.uint32(0xFFFFFFE0)            # garbage in bits >= k of both factors

@@ -4,13 +4,15 @@ Some users of this library run under a fixed memory budget: a server that carved
 start-up, or a plug-in that was never given the right to call cudaMalloc (which can also block, or
 fail half-way through a request).  For them lrbi_masked_gemm_static keeps the K-split partial sums in
 an 8 MiB array that is part of the library itself.  This file checks, through the C ABI, that it gives
-the same Y as lrbi_masked_gemm, twice in a row (the second call finds the first call's leftovers in
-the shared array), and that it refuses, without launching, what does not fit.  It is collected last on
+the same Y as lrbi_masked_gemm and as the CPU oracle, twice in a row (the second call finds the first
+call's leftovers in the shared array), that the device's free memory does not move while it is called
+again and again, and that it refuses, without launching, what does not fit.  It is collected last on
 purpose, so a run that stops at the first failure has already been through every other test.
 """
 import numpy as np
 import pytest
 
+import oracle
 from paper_1905_05686_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -41,7 +43,12 @@ def test_static_scratch_entry_point_matches_the_allocating_one_twice(y_dtype):
     B, W, ip, iz, X = _inputs(layer, batch)
     need = B.masked_gemm_static_bytes(layer, batch)
     assert 0 < need <= B.STATIC_SCRATCH_BYTES, "this shape is meant to split K and to fit the fixed array"
+    assert B.masked_gemm_plan(layer, batch, B.ALGO_TENSOR).k_splits > 1
     want = B.lrbi_masked_gemm(layer, W, ip, iz, X, y_dtype=dt, algo=B.ALGO_TENSOR).float().cpu().numpy().astype(np.float64)
+    Ip, Iz = synth.make_factors(layer)
+    ref = oracle.masked_gemm(synth.make_weights(layer), oracle.decode_mask(Ip, Iz, layer.rows, layer.cols),
+                             synth.make_activations(layer, batch))
+    assert rel_fro(want, ref) <= (TOL if y_dtype == "bf16" else 2e-5)
     for call in range(2):
         # a different batch in between leaves other partial sums behind in the shared array
         if call == 1:
@@ -53,7 +60,27 @@ def test_static_scratch_entry_point_matches_the_allocating_one_twice(y_dtype):
         got = Y.float().cpu().numpy().astype(np.float64)
         assert np.isfinite(got).all()
         assert rel_fro(got, want) <= TOL, (call, rel_fro(got, want))
+        assert rel_fro(got, ref) <= (TOL if y_dtype == "bf16" else 2e-5), (call, rel_fro(got, ref))
     assert B.device_status() == 0
+
+
+def test_static_scratch_entry_point_leaves_free_memory_alone():
+    """After one warm-up call (module load, address look-up) the driver's count of free device bytes does
+    not move, however often the entry point is called and whatever batch it is given."""
+    layer = synth.Layer("noalloc", 1024, 4608, 512, 512, 32, 0.09, 0.01)
+    B, W, ip, iz, X16 = _inputs(layer, 16)
+    _, _, _, _, X48 = _inputs(layer, 48, seed_shift=3)
+    Y16 = torch.empty((16, layer.rows), dtype=torch.bfloat16, device="cuda")
+    Y48 = torch.empty((48, layer.rows), dtype=torch.float32, device="cuda")
+    B.lrbi_masked_gemm_static(layer, W, ip, iz, X16, Y16)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(20):
+        B.lrbi_masked_gemm_static(layer, W, ip, iz, X16, Y16)
+        B.lrbi_masked_gemm_static(layer, W, ip, iz, X48, Y48)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
 
 
 def test_static_scratch_entry_point_needs_no_scratch_for_large_batches():
@@ -64,7 +91,12 @@ def test_static_scratch_entry_point_needs_no_scratch_for_large_batches():
     want = B.lrbi_masked_gemm(layer, W, ip, iz, X, algo=B.ALGO_TENSOR).float().cpu().numpy().astype(np.float64)
     Y = torch.empty((batch, layer.rows), dtype=torch.bfloat16, device="cuda")
     B.lrbi_masked_gemm_static(layer, W, ip, iz, X, Y)
-    assert rel_fro(Y.float().cpu().numpy().astype(np.float64), want) <= TOL
+    got = Y.float().cpu().numpy().astype(np.float64)
+    assert rel_fro(got, want) <= TOL
+    Ip, Iz = synth.make_factors(layer)
+    ref = oracle.masked_gemm(synth.make_weights(layer), oracle.decode_mask(Ip, Iz, layer.rows, layer.cols),
+                             synth.make_activations(layer, batch))
+    assert rel_fro(got, ref) <= TOL
 
 
 def test_static_scratch_entry_point_refuses_what_does_not_fit():
