@@ -36,6 +36,7 @@
 // TMA thread drains (bounded) the copies it has in flight, and tensor memory is freed before exit.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "lrbi_common.cuh"
@@ -304,7 +305,7 @@ __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
 // one tensor core pass instead of two.  Two such blocks are resident per SM (three stages each), so
 // one block's epilogue and panel hand-overs overlap the other's MMAs.
 template <int BN, int PW, bool PAIR>
-__global__ void __launch_bounds__(TC_THREADS, 2)
+__global__ void __launch_bounds__(TC_THREADS, BN > 256 ? 1 : 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
@@ -314,6 +315,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // rows of X this CTA loads per stage
     constexpr int B_STAGE_BYTES = B_ROWS * TC_BK * 2;
     constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    // Pair mode, BN = 512: two accumulators of 256 batch columns fill the 512 columns of tensor memory.
+    // A pruned W stage then feeds two MMAs, so decode and pruning are amortised over twice the tensor work.
+    // Accumulator a covers batch rows b0 + 256 a ...; CTA `rank` loads the 128 rows b0 + 256 a + 128 rank ...
+    // of it as box a of its B stage.
+    constexpr int NACC = PAIR ? BN / 256 : 1;
+    constexpr int XBOX_ROWS = PAIR ? 128 : BN;          // rows of one TMA box of X
+    constexpr int MMA_N = PAIR ? 256 : BN;
+    static_assert(!PAIR || BN == 256 || BN == 512, "pair mode: one or two 256-column accumulators");
     constexpr int KBP = PW / 2;                          // K blocks per panel
     uint8_t *a_base = smem;
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
@@ -386,7 +395,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) break;
                 mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES + TC_A_STAGE_BYTES);
                 tma_load_2d(a_base + s * TC_A_STAGE_BYTES, &w_map, &ctl->full[s], (kb_begin + it) * TC_BK, o0);
-                tma_load_2d(b_base + s * B_STAGE_BYTES, &x_map, &ctl->full[s], (kb_begin + it) * TC_BK, b0 + (int)rank * B_ROWS);
+#pragma unroll
+                for (int a = 0; a < NACC; ++a)
+                    tma_load_2d(b_base + s * B_STAGE_BYTES + a * (XBOX_ROWS * TC_BK * 2), &x_map, &ctl->full[s],
+                                (kb_begin + it) * TC_BK, b0 + a * 256 + (int)rank * XBOX_ROWS);
                 issued = true;
                 if (++s == stages) { s = 0; parity ^= 1; }
             }
@@ -401,7 +413,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = PAIR ? make_idesc(BN, 2 * TC_BM) : make_idesc(BN);
+            constexpr uint32_t idesc = PAIR ? make_idesc(MMA_N, 2 * TC_BM) : make_idesc(MMA_N);
             bool ok = true;
             int s = 0;
             uint32_t parity = 0;
@@ -415,8 +427,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
 #pragma unroll
                 for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
                     // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in address units
-                    if (PAIR) umma2_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
-                    else umma_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
+                    if (PAIR) {
+#pragma unroll
+                        for (int a = 0; a < NACC; ++a)   // box a of the B stage -> accumulator a (256 columns further)
+                            umma2_bf16(tmem_d + (uint32_t)(a * 256), da + (uint64_t)(2 * k4),
+                                       db + (uint64_t)(a * ((XBOX_ROWS * TC_BK * 2) >> 4) + 2 * k4), idesc, (it | k4) ? 1u : 0u);
+                    } else {
+                        umma_bf16(tmem_d, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), idesc, (it | k4) ? 1u : 0u);
+                    }
                 }
                 // frees the stage (in both CTAs of a pair) when these MMAs have read it
                 if (PAIR) umma2_commit_both(&ctl->empty[s]); else umma_commit(&ctl->empty[s]);
@@ -791,6 +809,12 @@ static bool make_tc_plan(const Geo &g, int batch, int sm_count, TcPlan *out)
     // (a layer with few rows): then single CTAs with 128-row batch tiles give twice as many blocks
     p.pair = use_pairs(g, batch, sm_count);
     p.bn = batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : (batch <= 128 || !p.pair) ? 128 : 256;
+    if (p.pair) {
+        // two accumulators per pair (512 batch columns) when that still leaves several waves of blocks
+        const long long blocks512 = 2LL * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) * ((batch + 511) / 512);
+        if (blocks512 >= 4LL * sm_count) p.bn = 512;
+        if (const char *e = getenv("LRBI_TC_BN")) p.bn = atoi(e);   // EXPERIMENT ONLY
+    }
     // index words per panel row: 256-column panels when every panel then lies inside one tile
     p.pw = (g.gc == 1 || (g.tn % 256) == 0) ? 8 : 2;
     const int nkb = (g.cols + TC_BK - 1) / TC_BK;
@@ -848,7 +872,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.cols, (cuuint64_t)batch};
     const cuuint64_t strides[1] = {(cuuint64_t)g.cols * 2};
-    const cuuint32_t box[2] = {TC_BK, PAIR ? BN / 2 : BN};
+    const cuuint32_t box[2] = {TC_BK, PAIR ? 128 : BN};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -928,6 +952,7 @@ static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, c
     LRBI_TC_CASE(64, 8, false) LRBI_TC_CASE(64, 2, false)
     LRBI_TC_CASE(128, 8, false) LRBI_TC_CASE(128, 2, false)
     LRBI_TC_CASE(256, 8, true) LRBI_TC_CASE(256, 2, true)
+    LRBI_TC_CASE(512, 8, true) LRBI_TC_CASE(512, 2, true)
 #undef LRBI_TC_CASE
     return LRBI_ERR_UNSUPPORTED;
 }
