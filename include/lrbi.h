@@ -97,7 +97,11 @@ enum {
     LRBI_ALGO_DECODE_BALLOT = 4, /* decode: one __ballot_sync per 32-bit mask word             */
     LRBI_ALGO_DECODE_PLANES = 5, /* decode: Iz transposed into bit-planes, OR per 32 columns (variant by size) */
     LRBI_ALGO_DECODE_PLANES_WIDE = 6, /* decode: the 1024-column bit-plane variant, whatever the mask size */
-    LRBI_ALGO_STREAM = 7     /* batch <= 32, bandwidth-bound, warp-level tensor-core MMAs              */
+    LRBI_ALGO_STREAM = 7,    /* batch <= 32, bandwidth-bound, warp-level tensor-core MMAs              */
+    /* The next two force an instantiation that LRBI_ALGO_TENSOR otherwise picks from the problem size
+       (any shape LRBI_ALGO_TENSOR covers; small problems just leave most of a tile empty). */
+    LRBI_ALGO_TENSOR_PAIR = 8,  /* tcgen05 CTA pairs (cta_group::2), 256 rows x 256 batch rows per pair  */
+    LRBI_ALGO_TENSOR_PAIR2 = 9  /* CTA pairs with two accumulators: 256 rows x 512 batch rows per pair   */
 };
 
 /* Element counts of the packed arrays for a layout (0 if the layout is invalid). */
@@ -127,7 +131,8 @@ LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t 
  *   W      device, bf16 bit patterns, [rows][cols] row-major
  *   X      device, bf16 bit patterns, [batch][cols] row-major
  *   Y      device, [batch][rows] row-major, bf16 (round to nearest even) or fp32 per y_dtype
- *   algo   LRBI_ALGO_AUTO, _GENERIC, _GEMV (batch <= 8), _STREAM (batch <= 32) or _TENSOR; a kernel that does not
+ *   algo   LRBI_ALGO_AUTO, _GENERIC, _GEMV (batch <= 8), _STREAM (batch <= 32), _TENSOR, _TENSOR_PAIR or
+ *          _TENSOR_PAIR2; a kernel that does not
  *          cover the shape returns LRBI_ERR_UNSUPPORTED and launches nothing.
  * The tensor-core path may split the reduction over several thread blocks; it then keeps
  * fp32 partial sums in a library-owned device buffer that grows (cudaMalloc) on the first
@@ -155,7 +160,7 @@ LRBI_API lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t 
  *
  *   - If splits * batch * rows * 4 bytes exceeds that array the call returns LRBI_ERR_TOO_LARGE
  *     and launches nothing (lrbi_masked_gemm_static_bytes tells the need in advance; 0 = no
- *     scratch needed).  Large batches do not split K and need none.
+ *     scratch needed).  Problems with enough output tiles to fill the GPU do not split K and need none.
  *   - It calls no cudaMalloc, cudaFree or any other allocating routine.
  *   - The first call on a device looks up the array's device address (once per device, with that
  *     device current) and caches it; make that first call before starting any stream capture.
@@ -199,7 +204,7 @@ LRBI_API int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batc
  */
 typedef struct {
     int32_t algo;          /* the LRBI_ALGO_* value that runs (LRBI_ALGO_AUTO resolved)             */
-    int32_t batch_tile;    /* batch rows per output tile                                            */
+    int32_t batch_tile;    /* batch rows per output tile (512: a CTA pair with two accumulators)    */
     int32_t cta_pair;      /* 1: two CTAs of a cluster share a 256-row tile (tcgen05 cta_group::2)  */
     int32_t panel_columns; /* columns of the index decoded per step inside the kernel (256 or 64)   */
     int32_t k_splits;      /* thread blocks along the reduction; > 1 means fp32 partial sums + a second kernel */

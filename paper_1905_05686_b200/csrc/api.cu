@@ -149,6 +149,8 @@ lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const
     case LRBI_ALGO_GEMV: return launch_gemv(g, W, ip, iz, X, batch, Y, y_dtype, s);
     case LRBI_ALGO_STREAM: return launch_stream_mma(g, W, ip, iz, X, batch, Y, y_dtype, s);
     case LRBI_ALGO_TENSOR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s);
+    case LRBI_ALGO_TENSOR_PAIR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 1);
+    case LRBI_ALGO_TENSOR_PAIR2: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 2);
     default: return LRBI_ERR_INVALID_ARG;
     }
 }
@@ -199,7 +201,9 @@ lrbi_status lrbi_masked_gemm_plan(const lrbi_layout *layout, int32_t batch, int3
     case LRBI_ALGO_GENERIC: return LRBI_OK;
     case LRBI_ALGO_GEMV: return gemv_supported(g, batch) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
     case LRBI_ALGO_STREAM: return stream_mma_supported(g, batch) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
-    case LRBI_ALGO_TENSOR: return gemm_tc_plan(g, batch, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    case LRBI_ALGO_TENSOR: return gemm_tc_plan(g, batch, 0, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    case LRBI_ALGO_TENSOR_PAIR: return gemm_tc_plan(g, batch, 1, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    case LRBI_ALGO_TENSOR_PAIR2: return gemm_tc_plan(g, batch, 2, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
     default: return LRBI_ERR_INVALID_ARG;
     }
 }

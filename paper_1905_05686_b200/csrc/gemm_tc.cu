@@ -36,19 +36,22 @@
 // TMA thread drains (bounded) the copies it has in flight, and tensor memory is freed before exit.
 #include <cuda.h>
 
-#include <cstdlib>
 #include <mutex>
 
 #include "lrbi_common.cuh"
 
 namespace lrbi {
 
-constexpr int TC_THREADS = 448;
+constexpr int TC_THREADS = 448;               // with one group of decoder warps; a second group adds 128
 constexpr int TC_BM = 128;                 // rows of W per block (MMA M)
 constexpr int TC_BK = 64;                  // columns per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_A_STAGE_BYTES = TC_BM * TC_BK * 2;
 constexpr int TC_MASK_WARPS = 8;           // warps 2-9: prune the W tile of each stage, then run the epilogue
 constexpr int TC_DECODE_WARPS = 4;         // warps 10-13: decode the index one panel ahead
+// Two-accumulator blocks (BN = 512) run a second group of decoder warps (14-17): group g decodes the panels
+// with P % 2 == g into index buffer g, so a panel may take two panels' worth of pruning time.
+__host__ __device__ constexpr int tc_decode_groups(int bn) { return bn > 256 ? 2 : 1; }
+__host__ __device__ constexpr int tc_threads(int bn) { return TC_THREADS + (tc_decode_groups(bn) - 1) * TC_DECODE_WARPS * 32; }
 constexpr long long TC_WAIT_LIMIT_CYCLES = 4000000000ll;          // about 2 s of SM clock
 constexpr uint32_t TC_SUSPEND_HINT_NS = 20000u;                   // a waiting thread may sleep this long per try
 
@@ -72,7 +75,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(TC_SUSPEND_HINT_NS) : "memory");
     return ok != 0;
@@ -179,7 +182,7 @@ __device__ __forceinline__ void mbar_arrive_remote(uint64_t *bar, uint32_t rank)
 {
     uint32_t remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
@@ -255,14 +258,13 @@ __device__ __forceinline__ void stage_panel_factors(const Geo &g, const uint32_t
 // Shared-memory bookkeeping that follows the operand stages.
 struct TcCtl {
     uint64_t full[8];        // TMA copies of a stage have landed
-    uint64_t masked[8];      // ... and its W tile has been pruned in place
-    uint64_t peer_masked[8]; // pair mode, leader CTA: the other CTA's stage is pruned too
+    uint64_t masked[8];      // ... and its W tile has been pruned in place (leader of a pair: in both CTAs)
     uint64_t empty[8];       // the MMAs that read the stage have completed
     uint64_t accum;
     uint64_t epi;            // the eight pruning warps meet here before the epilogue's copy-out
     uint64_t bits_ready[2];  // decoders -> pruners: the index bits of a panel are in buffer b
     uint64_t bits_free[2];   // pruners -> decoders: buffer b may be overwritten
-    uint64_t dsync;          // the four decoder warps meet here once per panel
+    uint64_t dsync[2];       // the four warps of a decoder group meet here twice per panel
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -294,6 +296,12 @@ __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
     return w;
 }
 
+// Decoder group of a thread (0 for every thread that is not in the second group).
+__device__ __forceinline__ int warp_of_thread_decoder_group(unsigned tid)
+{
+    return tid >= (unsigned)TC_THREADS ? 1 : 0;
+}
+
 // grid = (batch tiles, row tiles of 128, K splits).  When gridDim.z > 1 the block writes fp32
 // partial sums to `partials` [split][batch][rows]; a second kernel adds them up.
 // PW = 32-bit index words per row of a panel (8: 256-column panels, 2: 64-column panels).
@@ -305,7 +313,7 @@ __device__ __forceinline__ uint4 prune_chunk(uint4 w, uint32_t bits, int j)
 // one tensor core pass instead of two.  Two such blocks are resident per SM (three stages each), so
 // one block's epilogue and panel hand-overs overlap the other's MMAs.
 template <int BN, int PW, bool PAIR>
-__global__ void __launch_bounds__(TC_THREADS, BN > 256 ? 1 : 2)
+__global__ void __launch_bounds__(tc_threads(BN), BN > 256 ? 1 : 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
@@ -328,10 +336,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
     constexpr int PWS = PW == 8 ? 12 : PW;               // words between planes (padded: conflict-free 16-byte reads)
     uint32_t *row_bits = reinterpret_cast<uint32_t *>(b_base + (size_t)stages * B_STAGE_BYTES);   // [2][128][PW]
-    uint32_t *planes = row_bits + 2 * TC_BM * PW;                                                  // [kw*32][PWS]
-    uint32_t *iz_stage = planes + g.kw * 32 * PWS;                                                 // [PW*32][kw]
-    uint32_t *ip_stage = iz_stage + PW * 32 * g.kw;                                                // [128][kw]
-    TcCtl *ctl = reinterpret_cast<TcCtl *>(ip_stage + TC_BM * g.kw);
+    constexpr int NDG = tc_decode_groups(BN);            // groups of decoder warps
+    // per decoder group: planes [kw*32][PWS], iz_stage [PW*32][kw], ip_stage [128][kw]
+    const int dgroup_words = g.kw * 32 * PWS + PW * 32 * g.kw + TC_BM * g.kw;
+    const int dgrp = warp_of_thread_decoder_group(threadIdx.x);
+    uint32_t *planes = row_bits + 2 * TC_BM * PW + dgrp * dgroup_words;
+    uint32_t *iz_stage = planes + g.kw * 32 * PWS;
+    uint32_t *ip_stage = iz_stage + PW * 32 * g.kw;
+    TcCtl *ctl = reinterpret_cast<TcCtl *>(row_bits + 2 * TC_BM * PW + NDG * dgroup_words);
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -351,9 +363,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
 
     // Long-latency requests first: the decoder warps ask for the factor words of their first panel, one
     // thread warms the TMA descriptors; both overlap the barrier and tensor-memory set-up below.
-    if (warp >= 2 + TC_MASK_WARPS)
-        stage_panel_factors(g, ip, iz, iz_stage, ip_stage, PW * 32, kb_begin * TC_BK, o0,
-                            threadIdx.x - (2 + TC_MASK_WARPS) * 32, TC_DECODE_WARPS * 32);
+    if (warp >= 2 + TC_MASK_WARPS && dgrp * KBP < nkb)   // group g starts with panel g
+        stage_panel_factors(g, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + dgrp * KBP) * TC_BK, o0,
+                            (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1), TC_DECODE_WARPS * 32);
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&w_map) : "memory");
@@ -361,8 +373,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->masked[s], TC_MASK_WARPS);
-            mbar_init(&ctl->peer_masked[s], 1);
+            // leader of a pair: its stage is ready when its own eight pruning warps and the other CTA's relay have arrived
+            mbar_init(&ctl->masked[s], TC_MASK_WARPS + ((PAIR && rank == 0) ? 1 : 0));
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum, 1);
@@ -371,7 +383,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             mbar_init(&ctl->bits_ready[b], TC_DECODE_WARPS);
             mbar_init(&ctl->bits_free[b], TC_MASK_WARPS);
         }
-        mbar_init(&ctl->dsync, TC_DECODE_WARPS);
+        for (int b = 0; b < 2; ++b) mbar_init(&ctl->dsync[b], TC_DECODE_WARPS);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -419,7 +431,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             uint32_t parity = 0;
             for (int it = 0; it < nkb && ok; ++it) {
                 ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
-                if (ok && PAIR) ok = mbar_wait(&ctl->peer_masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t da = make_sw128_desc(smem_u32(a_base + s * TC_A_STAGE_BYTES));
@@ -452,13 +463,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             for (int it = 0; it < nkb && ok; ++it) {
                 ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
-                mbar_arrive_remote(&ctl->peer_masked[s], 0);
+                mbar_arrive_remote(&ctl->masked[s], 0);
                 if (++s == stages) { s = 0; parity ^= 1; }
             }
         }
     } else if (warp >= 2 + TC_MASK_WARPS) {
         // ------------------------------------------------------------- index decoders
-        const int dt = threadIdx.x - (2 + TC_MASK_WARPS) * 32;   // 0..127: row of the block this thread decodes
+        const int dt = (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1);   // 0..127: row of the block this thread decodes
         const int dw = dt >> 5;                         // decoder warp 0..3
         const uint32_t tail = tail_mask(g.k);
         const int tr = o0 / g.tm;                       // the 128 rows lie in one tile row
@@ -477,13 +488,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         bool ok = true;
         auto dsync = [&]() {                            // the four decoder warps meet (bounded wait)
             __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->dsync);
-            ok = mbar_wait(&ctl->dsync, dsync_parity, abort_flag, status, DEV_TIMEOUT_EMPTY);
+            if (lane == 0) mbar_arrive(&ctl->dsync[dgrp]);
+            ok = mbar_wait(&ctl->dsync[dgrp], dsync_parity, abort_flag, status, DEV_TIMEOUT_EMPTY);
             dsync_parity ^= 1;
         };
 
-        // (panel 0 was requested at kernel entry)
-        for (int P = 0; P < npanels && ok; ++P) {
+        // (the group's first panel was requested at kernel entry)
+        for (int P = dgrp; P < npanels && ok; P += NDG) {
             const int buf = P & 1;
             uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
             const int c0 = (kb_begin + P * KBP) * TC_BK;
@@ -517,7 +528,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             }
             dsync();                                     // planes complete, factor staging consumed
             if (!ok) break;
-            stage_factors(P + 1);                        // next panel's factor words start their trip now
+            stage_factors(P + NDG);                      // the group's next panel: its factor words start their trip now
             // the pruning warps must be done with the panel that used this buffer two panels ago
             ok = mbar_wait(&ctl->bits_free[buf], ((P >> 1) & 1) ^ 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
             if (!ok) break;
@@ -794,38 +805,49 @@ struct TcPlan {
     size_t scratch;      // bytes of fp32 partial sums (0 when K is not split)
 };
 
-static bool use_pairs(const Geo &g, int batch, int sm_count)
-{
-    if (batch <= 128) return false;
-    const long long pair_blocks = 2LL * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) * ((batch + 255) / 256);
-    return pair_blocks * 2 >= 3LL * sm_count;
-}
-
-static bool make_tc_plan(const Geo &g, int batch, int sm_count, TcPlan *out)
+// `force`: 0 = choose by shape; 1 = CTA pairs with one accumulator (256 batch columns per pair);
+// 2 = CTA pairs with two accumulators (512 batch columns per pair).
+static bool make_tc_plan(const Geo &g, int batch, int sm_count, int force, TcPlan *out)
 {
     if (!gemm_tc_supported(g, batch)) return false;
     TcPlan p;
-    // large batch: CTA pairs share each X tile, unless there are too few pairs of tiles to fill the chip
-    // (a layer with few rows): then single CTAs with 128-row batch tiles give twice as many blocks
-    p.pair = use_pairs(g, batch, sm_count);
-    p.bn = batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : (batch <= 128 || !p.pair) ? 128 : 256;
-    if (p.pair) {
-        // two accumulators per pair (512 batch columns) when that still leaves several waves of blocks
-        const long long blocks512 = 2LL * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) * ((batch + 511) / 512);
-        if (blocks512 >= 4LL * sm_count) p.bn = 512;
-        if (const char *e = getenv("LRBI_TC_BN")) p.bn = atoi(e);   // EXPERIMENT ONLY
-    }
+    // Measured on B200 (K = 4096, microseconds; single CTAs with 128-column tiles / pairs with one / with two
+    // accumulators): 1024 x 4096 outputs 88 / 68 / 64; 4096 x 4096 283 / 174 / 125; 16384 x 4096 (the FFN
+    // layer) - / 568 / 408.  So: pairs whenever there are two 128-row blocks to pair and more than 128
+    // batch rows, two accumulators whenever the batch has more than 256 rows.
+    p.pair = force ? true : (batch > 128 && g.rows > TC_BM);
+    p.bn = batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : 128;
+    if (p.pair) p.bn = force == 1 ? 256 : force == 2 ? 512 : (batch > 256 ? 512 : 256);
     // index words per panel row: 256-column panels when every panel then lies inside one tile
     p.pw = (g.gc == 1 || (g.tn % 256) == 0) ? 8 : 2;
     const int nkb = (g.cols + TC_BK - 1) / TC_BK;
     p.row_blocks = p.pair ? 2 * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) : (g.rows + TC_BM - 1) / TC_BM;
-    const int tiles = ((batch + p.bn - 1) / p.bn) * p.row_blocks;
-    // split K when the output tiles alone cannot occupy the chip (small batch: bandwidth-bound)
+    const long long tiles = (long long)((batch + p.bn - 1) / p.bn) * p.row_blocks;
+    // Split K when the output tiles alone cannot occupy the chip.
     int splits = 1;
-    if (batch <= p.bn && tiles < 2 * sm_count) {      // one batch tile: the small-batch, bandwidth-bound case
-        splits = (2 * sm_count + tiles - 1) / tiles;
-        splits = splits > nkb / 4 ? (nkb / 4 > 0 ? nkb / 4 : 1) : splits;   // at least 4 K blocks per split
-        if (splits > 32) splits = 32;
+    if (!p.pair) {
+        if (batch <= p.bn && tiles < 2 * sm_count) {  // one batch tile: the small-batch, bandwidth-bound case
+            splits = (int)((2 * sm_count + tiles - 1) / tiles);
+            splits = splits > nkb / 4 ? (nkb / 4 > 0 ? nkb / 4 : 1) : splits;   // at least 4 K blocks per split
+            if (splits > 32) splits = 32;
+        }
+    } else {
+        // A lone block advances about one K block per microsecond (its ring of stages is bound by latency, not
+        // by the tensor pipe), so cutting K pays when blocks are few -- as long as writing and re-reading the
+        // fp32 partial sums (about 5 bytes per nanosecond) costs less than half of the time it saves.
+        const long long slots = (long long)sm_count * (p.bn == 512 ? 1 : 2);
+        if (tiles < slots) {
+            int sp = (int)(slots / tiles);
+            if (sp > nkb / 8) sp = nkb / 8;           // at least 8 K blocks per split
+            if (sp > 32) sp = 32;
+            while (sp > 1) {
+                const double partial_us = (double)sp * batch * g.rows * 8.0 / 5.0e6;
+                const double saved_us = (double)(nkb - (nkb + sp - 1) / sp);
+                if (partial_us <= 0.5 * saved_us) break;
+                --sp;
+            }
+            splits = sp < 1 ? 1 : sp;
+        }
     }
     int kb_per_split = (nkb + splits - 1) / splits;
     kb_per_split = (kb_per_split + 3) / 4 * 4;                               // splits start on panel boundaries
@@ -838,7 +860,8 @@ static bool make_tc_plan(const Geo &g, int batch, int sm_count, TcPlan *out)
     // overlap one's epilogue and hand-overs with the other's MMAs and double the copies in flight.
     // (an SM has 228 KB of shared memory; each resident block also reserves 1 KB)
     const size_t b_stage = (size_t)(p.pair ? p.bn / 2 : p.bn) * TC_BK * 2;
-    const size_t extras = (size_t)(2 * TC_BM * p.pw + g.kw * 32 * (p.pw == 8 ? 12 : p.pw) + p.pw * 32 * g.kw + TC_BM * g.kw) * 4 + sizeof(TcCtl);
+    const size_t dgroup_words = (size_t)g.kw * 32 * (p.pw == 8 ? 12 : p.pw) + (size_t)p.pw * 32 * g.kw + (size_t)TC_BM * g.kw;
+    const size_t extras = ((size_t)2 * TC_BM * p.pw + tc_decode_groups(p.bn) * dgroup_words) * 4 + sizeof(TcCtl);
     const size_t per_stage = TC_A_STAGE_BYTES + b_stage;
     const size_t half_sm = 113 * 1024, whole_sm = 224 * 1024;
     int stages = (int)((half_sm - extras) / per_stage);
@@ -901,7 +924,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     dim3 grid(PAIR ? 2 * nbt : nbt, (unsigned)(PAIR ? plan.row_blocks / 2 : plan.row_blocks), (unsigned)plan.splits);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(TC_THREADS);
+    cfg.blockDim = dim3(tc_threads(BN));
     cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -929,14 +952,14 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
 // `fixed_scratch` != nullptr: the caller forbids allocation, partial sums go there (fixed_bytes) or nowhere.
 static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s,
-                          float *fixed_scratch, size_t fixed_bytes)
+                          float *fixed_scratch, size_t fixed_bytes, int force = 0)
 {
     if (!gemm_tc_supported(g, batch)) return LRBI_ERR_UNSUPPORTED;    // shape errors come before device errors
     int dev = -1;
     const int sm_count = device_sm_count(&dev);
     if (dev < 0) return LRBI_ERR_CUDA;
     TcPlan plan;
-    if (!make_tc_plan(g, batch, sm_count, &plan)) return LRBI_ERR_UNSUPPORTED;
+    if (!make_tc_plan(g, batch, sm_count, force, &plan)) return LRBI_ERR_UNSUPPORTED;
     if (fixed_scratch && plan.scratch > fixed_bytes) return LRBI_ERR_TOO_LARGE;   // before any launch
     if (!device_status_ptr()) return LRBI_ERR_CUDA;
     float *partials = nullptr;
@@ -958,17 +981,17 @@ static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, c
 }
 
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s)
+                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force)
 {
-    return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, nullptr, 0);
+    return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, nullptr, 0, force);
 }
 
-bool gemm_tc_plan(const Geo &g, int batch, lrbi_gemm_plan *out)
+bool gemm_tc_plan(const Geo &g, int batch, int force, lrbi_gemm_plan *out)
 {
     int dev = -1;
     const int sm_count = device_sm_count(&dev);
     TcPlan p;
-    if (!make_tc_plan(g, batch, sm_count, &p)) return false;
+    if (!make_tc_plan(g, batch, sm_count, force, &p)) return false;
     out->batch_tile = p.bn;
     out->cta_pair = p.pair ? 1 : 0;
     out->panel_columns = p.pw * 32;
@@ -1006,7 +1029,7 @@ size_t gemm_tc_scratch_bytes(const Geo &g, int batch)
     int dev = -1;
     const int sm_count = device_sm_count(&dev);
     TcPlan p;
-    return make_tc_plan(g, batch, sm_count, &p) ? p.scratch : 0;
+    return make_tc_plan(g, batch, sm_count, 0, &p) ? p.scratch : 0;
 }
 
 lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,

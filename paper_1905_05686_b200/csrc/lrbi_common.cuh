@@ -127,14 +127,15 @@ lrbi_status launch_stream_mma(const Geo &g, const uint16_t *W, const uint32_t *i
                               const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 bool gemm_tc_supported(const Geo &g, int batch);
 // When it splits K the launcher keeps fp32 partial sums in the library-owned buffer of the device.
+// force: 0 = instantiation chosen by shape, 1 = CTA pairs (one accumulator), 2 = CTA pairs (two accumulators)
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force = 0);
 
 // Variant that keeps K-split partial sums in the library's fixed device array; allocates nothing.
 lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                                   const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 size_t gemm_tc_scratch_bytes(const Geo &g, int batch);   // fp32 partial sums the tensor-core path would keep
 lrbi_status launch_bounded_wait_selftest(unsigned limit_us, cudaStream_t s);
-bool gemm_tc_plan(const Geo &g, int batch, lrbi_gemm_plan *out);   // fills the tensor-core fields of the plan
+bool gemm_tc_plan(const Geo &g, int batch, int force, lrbi_gemm_plan *out);   // fills the tensor-core fields of the plan
 
 }  // namespace lrbi

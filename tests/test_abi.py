@@ -78,8 +78,10 @@ def test_plan_query_runs_without_a_device(lib):
     """The plan is host arithmetic: which instantiation of the tensor-core kernel a call would run."""
     from paper_1905_05686_b200 import synth
     p = lib.masked_gemm_plan(synth.CONFIGS["ffn_16384x4096"], 4096)
-    assert (p.algo, p.cta_pair, p.batch_tile, p.panel_columns, p.k_splits) == (lib.ALGO_TENSOR, 1, 256, 256, 1)
+    assert (p.algo, p.cta_pair, p.batch_tile, p.panel_columns, p.k_splits) == (lib.ALGO_TENSOR, 1, 512, 256, 1)
     assert p.scratch_bytes == 0 and p.stages >= 3
+    p = lib.masked_gemm_plan(synth.CONFIGS["ffn_16384x4096"], 4096, lib.ALGO_TENSOR_PAIR)
+    assert (p.cta_pair, p.batch_tile) == (1, 256)
     p = lib.masked_gemm_plan(synth.CONFIGS["alexnet_fc"], 16)
     assert p.algo == lib.ALGO_TENSOR and p.cta_pair == 0 and p.k_splits > 1
     assert p.scratch_bytes == p.k_splits * 16 * 4096 * 4

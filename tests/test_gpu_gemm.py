@@ -289,9 +289,10 @@ def test_ffn_config_full():
 
 
 # ------------------------------------------------------------------------------------------------
-# CTA-pair instantiations of the tensor-core kernel (the ones large layers run on): they are chosen
-# only when there are enough 256 x 256 output tiles to fill the chip, so these shapes are wide in the
-# batch and thin in K (the oracle stays under a second each).
+# CTA-pair instantiations of the tensor-core kernel (the ones large layers run on), with one accumulator
+# (256 batch rows per pair) and with two (512 batch rows per pair; the headline workload's kernel).  They
+# are forced through LRBI_ALGO_TENSOR_PAIR / _PAIR2 so that every shape below runs in both; the shapes are
+# wide in the batch and thin in K (the oracle stays under a second each).
 # ------------------------------------------------------------------------------------------------
 PAIR_SHAPES = [
     # rows, cols, tm, tn, k, batch
@@ -302,34 +303,54 @@ PAIR_SHAPES = [
     (512, 320, 256, 320, 256, 14300),    # rank 256: eight index words
     (1024, 512, 512, 256, 64, 7200),     # exact tiling in rows and K, ragged batch only
     (1000, 264, 1000, 264, 7, 7300),     # one tile, K = 4 blocks + 8 columns, rows tail of 232
+    (384, 1344, 128, 1344, 40, 700),     # five full panels and one of 64 columns: both decoder groups, odd panel count
+    (256, 2304, 128, 256, 16, 130),      # nine panels, batch just above one CTA's half of a 256-row accumulator
 ]
 
 
-def _pair_case(shape):
+def _pair_algos():
     b = _b()
+    return [(b.ALGO_TENSOR_PAIR, 256), (b.ALGO_TENSOR_PAIR2, 512)]
+
+
+@pytest.mark.parametrize("width", [256, 512])
+@pytest.mark.parametrize("shape", PAIR_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_cta_pair_kernel(shape, width):
+    b = _b()
+    algo = dict((w, a) for a, w in _pair_algos())[width]
     rows, cols, tm, tn, k, batch = shape
     L = synth.Layer("pair", rows, cols, tm, tn, k, 0.25, 0.05)
-    plan = b.masked_gemm_plan(L, batch, b.ALGO_TENSOR)
-    assert plan.cta_pair == 1 and plan.batch_tile == 256, "shape no longer reaches the CTA-pair kernel"
-    return L, plan
-
-
-@pytest.mark.parametrize("shape", PAIR_SHAPES, ids=lambda s: "x".join(map(str, s)))
-def test_cta_pair_kernel(shape):
-    b = _b()
-    L, plan = _pair_case(shape)
+    plan = b.masked_gemm_plan(L, batch, algo)
+    assert plan.cta_pair == 1 and plan.batch_tile == width
     assert plan.panel_columns == (256 if (L.grid[1] == 1 or L.tile_cols % 256 == 0) else 64)
-    c = Case(L, shape[5])
+    c = Case(L, batch)
     before = b.launch_count()
-    c.check_full(b.ALGO_TENSOR)                       # bf16 and fp32 output
-    assert b.launch_count() - before == 2             # one kernel per call: K is not split in pair mode
+    c.check_full(algo)                                # bf16 and fp32 output
+    assert b.launch_count() - before == 2 * (1 if plan.k_splits == 1 else 2)
 
 
-def test_cta_pair_kernel_one_hot_and_degenerate_masks():
+def test_auto_choice_reaches_both_pair_instantiations():
+    """What LRBI_ALGO_TENSOR picks by itself: pairs above 128 batch rows, two accumulators above 256."""
     b = _b()
+    L = synth.Layer("pair", 1024, 512, 512, 256, 64, 0.25, 0.05)
+    for batch, width in ((200, 256), (7200, 512)):
+        plan = b.masked_gemm_plan(L, batch, b.ALGO_TENSOR)
+        assert plan.cta_pair == 1 and plan.batch_tile == width
+        Case(L, batch).check_full(b.ALGO_TENSOR)
+    # few output tiles and a long reduction: K is split in pair mode too (fp32 partial sums, second kernel)
+    L = synth.Layer("pairsplit", 512, 4096, 256, 1024, 64, 0.25, 0.05)
+    plan = b.masked_gemm_plan(L, 300, b.ALGO_TENSOR)
+    assert plan.cta_pair == 1 and plan.k_splits > 1
+    Case(L, 300).check_full(b.ALGO_TENSOR)
+
+
+@pytest.mark.parametrize("width", [256, 512])
+def test_cta_pair_kernel_one_hot_and_degenerate_masks(width):
+    b = _b()
+    algo = dict((w, a) for a, w in _pair_algos())[width]
     shape = (712, 384, 128, 128, 16, 9300)
-    L, _ = _pair_case(shape)
-    batch = shape[5]
+    rows, cols, tm, tn, k, batch = shape
+    L = synth.Layer("pair", rows, cols, tm, tn, k, 0.25, 0.05)
     # one-hot activations return masked columns of W exactly
     c = Case(L, batch)
     cols_hit = (np.arange(batch) * 7 + 3) % L.cols
@@ -339,15 +360,15 @@ def test_cta_pair_kernel_one_hot_and_degenerate_masks():
     c.X = b.to_device_bf16(c.Xb)
     M = c.mask()
     want = (synth.bf16_bits_to_f32(c.Wb) * M)[:, cols_hit].T.astype(np.float64)
-    assert (c.run(b.ALGO_TENSOR) == want).all()
-    assert (c.run(b.ALGO_TENSOR, torch.float32) == want).all()
+    assert (c.run(algo) == want).all()
+    assert (c.run(algo, torch.float32) == want).all()
     # nothing kept / everything kept
     c = Case(L, batch, p=0.0)
-    assert not c.run(b.ALGO_TENSOR).any()
+    assert not c.run(algo).any()
     c = Case(L, batch, p=1.0)
     W = synth.bf16_bits_to_f32(c.Wb).astype(np.float64)
     Xf = synth.bf16_bits_to_f32(c.Xb).astype(np.float64)
-    assert rel_fro(c.run(b.ALGO_TENSOR, torch.float32), Xf @ W.T) <= TOL_F32
+    assert rel_fro(c.run(algo, torch.float32), Xf @ W.T) <= TOL_F32
     # NaN / Inf parked in pruned weights never reach Y
     c = Case(L, batch)
     M = c.mask()
@@ -355,7 +376,7 @@ def test_cta_pair_kernel_one_hot_and_degenerate_masks():
     Wb = c.Wb.copy()
     Wb[M == 0] = np.where(np.arange((M == 0).sum()) % 2 == 0, 0x7FC0, 0xFF80).astype(np.uint16)
     c.Wb, c.W = Wb, b.to_device_bf16(Wb)
-    got = c.run(b.ALGO_TENSOR)
+    got = c.run(algo)
     assert np.isfinite(got).all() and rel_fro(got, want) <= TOL
 
 
@@ -365,7 +386,7 @@ def test_bits_beyond_rank_are_ignored_by_every_gemm_kernel(k):
     b = _b()
     L = synth.Layer("pad", 256, 512, 128, 128, k, 0.25, 0.05)
     garbage = np.uint32((0xFFFFFFFF << (k % 32)) & 0xFFFFFFFF)
-    for batch, algos in ((4, (b.ALGO_GENERIC, b.ALGO_GEMV, b.ALGO_STREAM)), (40, (b.ALGO_TENSOR,)), (300, (b.ALGO_TENSOR,))):
+    for batch, algos in ((4, (b.ALGO_GENERIC, b.ALGO_GEMV, b.ALGO_STREAM)), (40, (b.ALGO_TENSOR,)), (300, (b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2))):
         c = Case(L, batch)
         want = c.oracle_full()
         ipw, izw = synth.pack_ip(c.Ip).reshape(-1, L.kw), synth.pack_iz(c.Iz).reshape(-1, L.kw)
