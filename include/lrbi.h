@@ -115,8 +115,9 @@ LRBI_API size_t lrbi_mask_words(const lrbi_layout *layout);      /* rows*ceil(co
  *   mask_out  device, rows x ceil(cols/32) uint32, row-major; bit (c % 32) of word c / 32
  *             of row r is Ia[r][c]; bits beyond `cols` in the last word of a row are 0.
  *   algo      LRBI_ALGO_AUTO, LRBI_ALGO_DECODE_BALLOT, LRBI_ALGO_DECODE_PLANES (needs
- *             tile_cols % 32 == 0) or LRBI_ALGO_DECODE_PLANES_WIDE (needs tile_cols % 128 == 0 and
- *             rank <= 256); a variant that does not cover the layout returns LRBI_ERR_UNSUPPORTED
+ *             tile_cols % 32 == 0) or LRBI_ALGO_DECODE_PLANES_WIDE (needs rank <= 256 and tiles of 128, 256,
+ *             512 or a multiple of 1024 columns, or a single tile column of a multiple of 128 columns);
+ *             a variant that does not cover the layout returns LRBI_ERR_UNSUPPORTED
  * Every word of mask_out is written; nothing else is.
  */
 LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t *ip, const uint32_t *iz,

@@ -111,8 +111,25 @@ def test_ragged_shapes_planes(shape):
     check(synth.Layer("rag", rows, cols, tm, tn, k, 0.2), _algo("planes"))
 
 
-@pytest.mark.parametrize("shape", [s for s in RAGGED if s[3] % 128 == 0 and s[4] <= 256] +
-                         [(4096, 4096, 256, 256, 8), (2100, 3072, 1050, 1024, 64), (600, 2304, 128, 256, 16)],
+def _wide_covers(s):
+    """tiles of 128, 256 or 512 columns, of a multiple of 1024 columns, or one tile column of a multiple of 128; rank <= 256"""
+    rows, cols, tm, tn, k = s
+    return k <= 256 and tn % 128 == 0 and (cols <= tn or tn % 1024 == 0 or tn in (128, 256, 512))
+
+
+def test_wide_variant_refuses_other_tile_widths():
+    b = _b()
+    L = synth.Layer("rag", 1300, 1536, 1300, 768, 40, 0.2)      # two tile columns of 768
+    Ip, Iz = synth.make_factors(L)
+    with pytest.raises(b.LrbiError) as e:
+        gpu_decode(L, Ip, Iz, b.ALGO_DECODE_PLANES_WIDE)
+    assert e.value.code == b.ERR_UNSUPPORTED
+    check(L, b.ALGO_AUTO)                                        # the automatic choice still covers it
+
+
+@pytest.mark.parametrize("shape", [s for s in RAGGED if _wide_covers(s)] +
+                         [(1300, 768, 1300, 768, 40), (700, 5120, 350, 512, 8), (300, 2304, 100, 256, 3), (5000, 8192, 2500, 1024, 5),
+                          (4096, 4096, 256, 256, 8), (2100, 3072, 1050, 1024, 64), (600, 2304, 128, 256, 16)],
                          ids=lambda s: "x".join(map(str, s)))
 def test_ragged_shapes_planes_wide(shape):
     rows, cols, tm, tn, k = shape
