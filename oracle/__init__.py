@@ -10,6 +10,11 @@ Functions (citations are to the paper):
   masked_gemm          Y = X (W .* Ia)^T with Ia as the masking layer (Sections 2, 2.2).
   masked_gemm_samples  the same two definitions evaluated only at chosen outputs.
   bf16_to_f64          exact widening of bf16 bit patterns.
+Inner loop of Algorithm 1 (Section 2.1), in lrbi_alg1_oracle.c and, for the search itself, below:
+  threshold            binary conversion of NMF factors, entry = 1 iff value >= T (sentence under Eq. 4).
+  index_cost           per tile: ones of I and of Ia, and Cost = sum of |W| where I = 1 and Ia = 0.
+  sz_from_eq7          the inversion of Eq. 7 printed under it.
+  threshold_for_sparsity, alg1_search   the S_p sweep with the S_z search, in the order of Algorithm 1.
 """
 from __future__ import annotations
 
@@ -21,16 +26,17 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "lrbi_oracle.c")
+_SRC2 = os.path.join(_HERE, "lrbi_alg1_oracle.c")
 _LIB = os.path.join(_HERE, "liblrbi_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (-O2, OpenMP). Returns the path of the .so."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC2)):
         tmp = _LIB + ".tmp.%d" % os.getpid()
         subprocess.run(
-            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", tmp, _SRC],
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", tmp, _SRC, _SRC2, "-lm"],
             check=True,
         )
         os.replace(tmp, _LIB)
@@ -50,6 +56,10 @@ def _load():
         lib.lrbi_oracle_masked_gemm_samples.restype = None
         lib.lrbi_oracle_bf16_to_f64.argtypes = [i64, vp, vp]
         lib.lrbi_oracle_bf16_to_f64.restype = None
+        lib.lrbi_oracle_threshold.argtypes = [i64, i64, vp, vp, vp]
+        lib.lrbi_oracle_threshold.restype = None
+        lib.lrbi_oracle_index_cost.argtypes = [i64] * 4 + [vp, ctypes.c_float] + [vp] * 5
+        lib.lrbi_oracle_index_cost.restype = None
         lib.lrbi_oracle_threads.argtypes = []
         lib.lrbi_oracle_threads.restype = ctypes.c_int
         _lib = lib
@@ -134,3 +144,100 @@ def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
     out = np.empty(bits.shape, dtype=np.float64)
     _load().lrbi_oracle_bf16_to_f64(bits.size, bits.ctypes.data, out.ctypes.data)
     return out
+
+
+# ------------------------------------------------------------------------------------------------
+# Inner loop of Algorithm 1 (Section 2.1)
+# ------------------------------------------------------------------------------------------------
+def threshold(values: np.ndarray, T) -> np.ndarray:
+    """Binary conversion of NMF factors: entry = 1 iff value >= threshold (sentence under Eq. 4).
+
+    values: float32 [ntiles, ...]; T: one threshold per tile (a scalar is used for every tile).
+    """
+    values = _c(values, np.float32)
+    ntiles = values.shape[0]
+    T = np.ascontiguousarray(np.broadcast_to(np.asarray(T, dtype=np.float32), (ntiles,)))
+    out = np.empty(values.shape, dtype=np.uint8)
+    _load().lrbi_oracle_threshold(ntiles, values[0].size, values.ctypes.data, T.ctypes.data, out.ctypes.data)
+    return out
+
+
+def index_cost(W_bits: np.ndarray, theta: float, Ia: np.ndarray, tm: int, tn: int):
+    """Per tile (row-major grid order): ones of I = (|W| >= theta), ones of Ia, positions with I = 1 and
+    Ia = 0, and Cost = the sum of |W| over those positions (the cost line of Algorithm 1)."""
+    W_bits = _c(W_bits, np.uint16)
+    Ia = _c(Ia, np.uint8)
+    rows, cols = W_bits.shape
+    if Ia.shape != (rows, cols):
+        raise ValueError("shape mismatch")
+    gr, gc = _grid(rows, cols, tm, tn)
+    kept_i, kept_a, lost = (np.empty(gr * gc, dtype=np.int64) for _ in range(3))
+    cost = np.empty(gr * gc, dtype=np.float64)
+    _load().lrbi_oracle_index_cost(rows, cols, tm, tn, W_bits.ctypes.data, ctypes.c_float(np.float32(theta)), Ia.ctypes.data,
+                                   kept_i.ctypes.data, kept_a.ctypes.data, lost.ctypes.data, cost.ctypes.data)
+    return kept_i, kept_a, lost, cost
+
+
+def sz_from_eq7(S: float, Sp: float, k: int) -> float:
+    """S_z = (S^(1/k) - S_p) / (1 - S_p), the inversion of Eq. 7 printed under it."""
+    return (S ** (1.0 / k) - Sp) / (1.0 - Sp)
+
+
+def threshold_for_sparsity(values: np.ndarray, sparsity: float) -> np.float32:
+    """The threshold that turns the fraction `sparsity` of the entries into zeros: with the entries sorted,
+    z = round(sparsity * n) of them must fall below it, so it is the z-th smallest value (+inf if z = n).
+    Ties at that value are all kept, so the sparsity reached can be lower.  (The paper converts "with
+    (S_p, S_z)" and gives no rule; this is the reading taken.)"""
+    v = np.sort(np.asarray(values, dtype=np.float32).ravel())
+    z = int(round(float(sparsity) * v.size))
+    z = min(max(z, 0), v.size)
+    return np.float32(np.inf) if z == v.size else v[z]
+
+
+def alg1_search(W_bits: np.ndarray, theta: float, Mp: np.ndarray, Mz: np.ndarray, sp_step: float = 0.05,
+                tol: float = 1e-3, max_iter: int = 24):
+    """Algorithm 1 for one matrix (one tile), from the NMF factors on: the S_p sweep, S_z from Eq. 7 then
+    adjusted by bisection until S_a is within `tol` of S, the cost of each candidate, the best one kept.
+
+    W_bits: uint16 [m, n]; Mp: float32 [m, k]; Mz: float32 [k, n]; the index I is |W| >= theta and the
+    target sparsity S is the sparsity of I.  The paper gives neither the step of the sweep, nor the
+    tolerance of "S_a ~ S", nor the number of adjustments: sp_step, tol and max_iter are this reading's.
+    Returns a dict with the best (Sp, Sz, Tp, Tz, cost, Sa) and the list of all candidates.
+    """
+    W_bits = _c(W_bits, np.uint16)
+    m, n = W_bits.shape
+    k = Mp.shape[1]
+    Mp = _c(Mp, np.float32).reshape(1, m, k)
+    Mz = _c(Mz, np.float32).reshape(1, k, n)
+    full = np.ones((m, n), dtype=np.uint8)
+    kept_i = index_cost(W_bits, theta, full, m, n)[0][0]
+    S = 1.0 - kept_i / float(m * n)
+    best, tried = None, []
+    nsteps = int(round(1.0 / sp_step))
+    for step in range(nsteps + 1):                       # "for S_p = 0.0 to 1.0"
+        Sp = min(step * sp_step, 1.0)
+        if Sp >= 1.0:
+            Sz0 = 0.0                                    # Ip empty: Ia is empty whatever Iz is
+        else:
+            Sz0 = min(max(sz_from_eq7(S, Sp, k), 0.0), 1.0)   # "compute S_z using Eq. 7"
+        Tp = threshold_for_sparsity(Mp, Sp)
+        Ip = threshold(Mp, Tp).reshape(1, 1, m, k)
+        lo, hi, Sz = 0.0, 1.0, Sz0
+        for it in range(max_iter):                       # "repeat ... until S_a ~ S"
+            Tz = threshold_for_sparsity(Mz, Sz)
+            Iz = threshold(Mz, Tz).reshape(1, 1, k, n)   # "convert (Mp, Mz) into (Ip, Iz) w/ (S_p, S_z)"
+            Ia = decode_mask(Ip, Iz, m, n)
+            _, kept_a, lost, cost = index_cost(W_bits, theta, Ia, m, n)
+            Sa = 1.0 - kept_a[0] / float(m * n)
+            if abs(Sa - S) <= tol:
+                break
+            if Sa > S:                                   # too sparse: keep more of Iz ("adjust S_z depending on S_a - S")
+                hi = Sz
+            else:
+                lo = Sz
+            Sz = 0.5 * (lo + hi)
+        cand = {"Sp": Sp, "Sz": Sz, "Tp": float(Tp), "Tz": float(Tz), "cost": float(cost[0]), "Sa": Sa, "lost": int(lost[0])}
+        tried.append(cand)
+        if best is None or best["cost"] > cand["cost"]:  # "if Cost_min > Cost"
+            best = cand
+    return {"S": S, "best": best, "tried": tried}
