@@ -195,6 +195,42 @@ LRBI_API lrbi_status lrbi_layer_forward_host(lrbi_layer *layer, const uint16_t *
                                     void *Y_host, int32_t y_dtype, int32_t algo);
 LRBI_API lrbi_status lrbi_layer_destroy(lrbi_layer *layer);
 
+/*
+ * Inner loop of Algorithm 1 (Section 2.1: "binary pruning-index-data matrix factorization").  The NMF of
+ * |W| and the search over S_p stay with the caller; these two calls are the steps the search repeats.
+ *
+ * lrbi_threshold_pack: binary conversion of the NMF factors (the sentence under Eq. 4; Eq. 4 -> Eq. 5),
+ *       (Ip)[i][l] = 1 if (Mp)[i][l] >= T_p else 0,     (Iz)[l][j] = 1 if (Mz)[l][j] >= T_z else 0,
+ * written in the packed factor format above.  Every tile is its own factorisation (Section 3.1) and has its
+ * own pair of thresholds.
+ *   mp   device, fp32, [GR*GC][tile_rows][rank]   row-major per tile
+ *   mz   device, fp32, [GR*GC][rank][tile_cols]   row-major per tile
+ *   tp, tz   device, fp32, [GR*GC]   thresholds of each tile (+inf gives an empty factor)
+ *   ip_out, iz_out   device, lrbi_packed_ip_words / lrbi_packed_iz_words words; bits >= rank are written as 0
+ *
+ * lrbi_index_cost: what the search looks at for one candidate (ip, iz), per tile, tiles in row-major grid order:
+ *   kept_i = number of ones of the magnitude index I = (|W| >= theta)            (Eq. 1 -> Eq. 2)
+ *   kept_a = number of ones of the decoded index Ia = Ip (x) Iz                  (Eq. 3; S_a = 1 - kept_a / size)
+ *   lost   = number of positions with I = 1 and Ia = 0
+ *   cost   = sum of |W| over those positions                                    (the Cost line of Algorithm 1)
+ * W is read once, Ia is decoded on the fly and never stored.  A NaN weight counts as pruned (I = 0).  cost is
+ * summed in fp32 per 8 weights and in fp64 beyond; blocks add to a tile's record with atomics, so the last bits
+ * of cost may differ between calls.
+ *   W    device, bf16 bit patterns, [rows][cols]
+ *   out  device, GR*GC records, 8-byte aligned; overwritten
+ * Only positions inside the matrix are counted (edge tiles are smaller).
+ */
+typedef struct {
+    uint64_t kept_i;
+    uint64_t kept_a;
+    uint64_t lost;
+    double cost;
+} lrbi_tile_cost;
+LRBI_API lrbi_status lrbi_threshold_pack(const lrbi_layout *layout, const float *mp, const float *mz, const float *tp,
+                                         const float *tz, uint32_t *ip_out, uint32_t *iz_out, void *stream);
+LRBI_API lrbi_status lrbi_index_cost(const lrbi_layout *layout, const uint16_t *W, float theta, const uint32_t *ip,
+                                     const uint32_t *iz, lrbi_tile_cost *out, void *stream);
+
 /* Which kernel LRBI_ALGO_AUTO would run for this layout and batch (an LRBI_ALGO_* value). */
 LRBI_API int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batch);
 

@@ -88,6 +88,10 @@ def lib():
         L.lrbi_last_device_error.restype = i32
         L.lrbi_selftest_bounded_wait.argtypes = [ctypes.c_uint32, vp]
         L.lrbi_selftest_bounded_wait.restype = i32
+        L.lrbi_threshold_pack.argtypes = [lp, vp, vp, vp, vp, vp, vp, vp]
+        L.lrbi_threshold_pack.restype = i32
+        L.lrbi_index_cost.argtypes = [lp, vp, ctypes.c_float, vp, vp, vp, vp]
+        L.lrbi_index_cost.restype = i32
         L.lrbi_launch_count.argtypes = []
         L.lrbi_launch_count.restype = ctypes.c_uint64
         L.lrbi_device_status.argtypes = [i32]
@@ -171,6 +175,55 @@ def lrbi_decode_mask(layer, ip: torch.Tensor, iz: torch.Tensor, mask_out: torch.
     if rc != OK:
         raise LrbiError(rc, "lrbi_decode_mask")
     return mask_out
+
+
+def lrbi_threshold_pack(layer, mp: torch.Tensor, mz: torch.Tensor, tp: torch.Tensor, tz: torch.Tensor, stream=None):
+    """Binary conversion of NMF factors into packed (ip, iz): mp [tiles, tm, k], mz [tiles, k, tn] fp32,
+    tp, tz [tiles] fp32 thresholds.  Returns the two packed int32 tensors."""
+    lay = Layout.of(layer)
+    L = lib()
+    gr, gc = -(-lay.rows // lay.tile_rows), -(-lay.cols // lay.tile_cols)
+    tiles = gr * gc
+    if mp.numel() != tiles * lay.tile_rows * lay.rank or mz.numel() != tiles * lay.rank * lay.tile_cols:
+        raise ValueError("factor sizes do not match the layout")
+    if tp.numel() != tiles or tz.numel() != tiles:
+        raise ValueError("one threshold pair per tile")
+    ip = torch.empty(L.lrbi_packed_ip_words(ctypes.byref(lay)), dtype=torch.int32, device=mp.device)
+    iz = torch.empty(L.lrbi_packed_iz_words(ctypes.byref(lay)), dtype=torch.int32, device=mp.device)
+    rc = L.lrbi_threshold_pack(ctypes.byref(lay), _dev(mp, torch.float32, "mp"), _dev(mz, torch.float32, "mz"),
+                               _dev(tp, torch.float32, "tp"), _dev(tz, torch.float32, "tz"),
+                               _dev(ip, torch.int32, "ip"), _dev(iz, torch.int32, "iz"), _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_threshold_pack")
+    return ip, iz
+
+
+def lrbi_index_cost(layer, W: torch.Tensor, theta: float, ip: torch.Tensor, iz: torch.Tensor, out: torch.Tensor | None = None,
+                    stream=None) -> torch.Tensor:
+    """Per-tile records (kept_i, kept_a, lost as int64 bit patterns, cost as the bits of a double): an int64
+    tensor [tiles, 4]; `tile_costs` turns it into numpy arrays."""
+    lay = Layout.of(layer)
+    L = lib()
+    if tuple(W.shape) != (lay.rows, lay.cols):
+        raise ValueError("W shape does not match the layout")
+    if ip.numel() != L.lrbi_packed_ip_words(ctypes.byref(lay)) or iz.numel() != L.lrbi_packed_iz_words(ctypes.byref(lay)):
+        raise ValueError("packed factor sizes do not match the layout")
+    tiles = (-(-lay.rows // lay.tile_rows)) * (-(-lay.cols // lay.tile_cols))
+    if out is None:
+        out = torch.empty((tiles, 4), dtype=torch.int64, device=W.device)
+    elif out.numel() != tiles * 4:
+        raise ValueError("out has the wrong size")
+    rc = L.lrbi_index_cost(ctypes.byref(lay), _dev(W, torch.bfloat16, "W"), ctypes.c_float(theta), _dev(ip, torch.int32, "ip"),
+                           _dev(iz, torch.int32, "iz"), _dev(out, torch.int64, "out"), _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_index_cost")
+    return out
+
+
+def tile_costs(out: torch.Tensor):
+    """(kept_i, kept_a, lost, cost) numpy arrays from the records lrbi_index_cost wrote."""
+    a = out.cpu().numpy()
+    return a[:, 0].copy(), a[:, 1].copy(), a[:, 2].copy(), a[:, 3].copy().view(np.float64)
 
 
 def lrbi_masked_gemm(layer, W: torch.Tensor, ip: torch.Tensor, iz: torch.Tensor, X: torch.Tensor,

@@ -173,6 +173,24 @@ size_t lrbi_masked_gemm_static_bytes(const lrbi_layout *layout, int32_t batch)
     return gemm_tc_supported(g, batch) ? gemm_tc_scratch_bytes(g, batch) : 0;
 }
 
+lrbi_status lrbi_threshold_pack(const lrbi_layout *layout, const float *mp, const float *mz, const float *tp,
+                                const float *tz, uint32_t *ip_out, uint32_t *iz_out, void *stream)
+{
+    if (!layout_ok(layout) || !mp || !mz || !tp || !tz || !ip_out || !iz_out) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(ip_out) || !aligned16(iz_out)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    return launch_threshold_pack(make_geo(*layout), mp, mz, tp, tz, ip_out, iz_out, static_cast<cudaStream_t>(stream));
+}
+
+lrbi_status lrbi_index_cost(const lrbi_layout *layout, const uint16_t *W, float theta, const uint32_t *ip,
+                            const uint32_t *iz, lrbi_tile_cost *out, void *stream)
+{
+    if (!layout_ok(layout) || !W || !ip || !iz || !out) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(ip) || !aligned16(iz) || (reinterpret_cast<uintptr_t>(out) & 7u)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    return launch_index_cost(make_geo(*layout), W, theta, ip, iz, out, static_cast<cudaStream_t>(stream));
+}
+
 uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t lrbi_device_status(int32_t clear)

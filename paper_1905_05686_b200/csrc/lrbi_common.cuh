@@ -138,4 +138,11 @@ size_t gemm_tc_scratch_bytes(const Geo &g, int batch);   // fp32 partial sums th
 lrbi_status launch_bounded_wait_selftest(unsigned limit_us, cudaStream_t s);
 bool gemm_tc_plan(const Geo &g, int batch, int force, lrbi_gemm_plan *out);   // fills the tensor-core fields of the plan
 
+
+// Inner loop of Algorithm 1.
+lrbi_status launch_threshold_pack(const Geo &g, const float *mp, const float *mz, const float *tp, const float *tz,
+                                  uint32_t *ip, uint32_t *iz, cudaStream_t s);
+lrbi_status launch_index_cost(const Geo &g, const uint16_t *W, float theta, const uint32_t *ip, const uint32_t *iz,
+                              lrbi_tile_cost *out, cudaStream_t s);
+
 }  // namespace lrbi
