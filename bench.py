@@ -32,8 +32,9 @@ L2_BYTES = 126 * 1024 * 1024
 # summarised under profiles/ (null for workloads without a capture of the current kernel)
 NCU_TRAFFIC_BYTES = {}
 # The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
+# batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
 OTHER_WORKLOADS = [("lenet_fc1", 32), ("decode_4096", 0), ("decode_32768", 0), ("alexnet_fc", 1), ("alexnet_fc", 16),
-                   ("alexnet_fc", 128), ("conv3x3_256", 12544)]
+                   ("alexnet_fc", 128), ("conv3x3_256", 12544), ("alexnet_fc", -1), ("ffn_16384x4096", -1)]
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -214,6 +215,8 @@ def roofline_of(workload, batch, work_bytes, work_flops, kernel_ms, peaks):
 def kernel_label(B, layer, batch):
     if not batch:
         return "decode"
+    if batch < 0:
+        return "index_cost"
     plan = B.masked_gemm_plan(layer, batch)
     name = B.ALGO_NAMES[plan.algo]
     if plan.algo == B.ALGO_TENSOR:
@@ -228,6 +231,7 @@ def setup_workload(B, workload, batch, rank=0):
 
     layer = synth.CONFIGS[workload]
     decode_only = not layer.batches
+    cost_only = batch is not None and batch < 0
     batch = 0 if decode_only else (batch or layer.batches[-1])
     Ip, Iz = synth.make_factors(layer)
     ipw, izw = synth.pack_ip(Ip), synth.pack_iz(Iz)
@@ -237,6 +241,13 @@ def setup_workload(B, workload, batch, rank=0):
         out = torch.empty((layer.rows, (layer.cols + 31) // 32), dtype=torch.int32, device="cuda")
         w.update(step=lambda: B.lrbi_decode_mask(layer, ip, iz, out), out=out,
                  work_bytes=decode_bytes(layer), work_flops=0)
+    elif cost_only:
+        gr, gc = layer.grid
+        W = B.to_device_bf16(synth.make_weights(layer))
+        out = torch.empty((gr * gc, 4), dtype=torch.int64, device="cuda")
+        theta = 1.5 * layer.w_std                       # |W| >= 1.5 sigma: about 13 % of a Gaussian layer kept
+        w.update(step=lambda: B.lrbi_index_cost(layer, W, theta, ip, iz, out=out), out=out, work_flops=0,
+                 work_bytes=2 * layer.rows * layer.cols + gr * gc * ((layer.tile_rows + layer.tile_cols) * layer.kw * 4 + 32))
     else:
         Wb = synth.make_weights(layer)
         xlayer = synth.Layer(**{**layer.__dict__, "seed": rank_seed(layer.seed, rank)})
@@ -408,7 +419,7 @@ def run_ours(args):
         flush2 = torch.zeros(256 * 1024 * 1024 // 4, dtype=torch.int32, device="cuda")
         for name, ob in OTHER_WORKLOADS:
             if name == args.workload and (ob == batch or not ob):
-                continue
+                continue                                  # the headline workload itself
             ow = setup_workload(B, name, ob)
             l0 = B.launch_count()
             ts = time_calls(ow["step"], args.other_steps, 3, flush2)

@@ -73,6 +73,26 @@ struct CostAcc {
     double cost;
 };
 
+// Eight consecutive weights (16 bytes) and the eight index bits of Ia that go with them: counts by popcount,
+// cost as a select-and-add in fp32 (eight terms; the caller carries it on in fp64).
+__device__ __forceinline__ void cost_chunk(const uint4 &v, uint32_t ia8, float theta, uint32_t &kept_i, uint32_t &kept_a,
+                                           uint32_t &lost, float &cost_f)
+{
+    const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+    uint32_t i8 = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const float m = __uint_as_float(((e & 1) ? ww[e >> 1] : (ww[e >> 1] << 16)) & 0x7FFF0000u);   // M = |W|
+        const bool i = m >= theta;                                          // I (false for NaN)
+        i8 |= i ? (1u << e) : 0u;
+        cost_f += (i && !((ia8 >> e) & 1u)) ? m : 0.f;
+    }
+    ia8 &= 0xFFu;
+    kept_i += __popc(i8);
+    kept_a += __popc(ia8);
+    lost += __popc(i8 & ~ia8);
+}
+
 __device__ __forceinline__ void cost_element(uint32_t wbits, bool ia, float theta, CostAcc &a, float &cost_f)
 {
     const float m = fabsf(__uint_as_float(wbits << 16));                     // M = |W|
@@ -110,33 +130,57 @@ index_cost_kernel(Geo g, const uint16_t *__restrict__ W, float theta, const uint
             a1_planes[(lb * 32 + lane) * tnw + w] = warp_transpose32(z, lane);
         }
         __syncthreads();
-        for (int i = i_begin + warp; i < i_end; i += A1_THREADS / 32) {
+        // A warp walks (row, 256-column chunk) pairs; a lane owns 8 consecutive columns of a chunk.  The weights
+        // of the next pair are requested before the current one is evaluated.
+        const int nch = (ncols + 255) >> 8;
+        const int nrows_w = i_begin + warp < i_end ? (i_end - i_begin - warp + A1_THREADS / 32 - 1) / (A1_THREADS / 32) : 0;
+        const uint16_t *wtile = W + (size_t)(tr * g.tm) * g.cols + (size_t)tc * g.tn;
+        auto load_w = [&](int j, int ch) {
+            const int c = ch * 256 + lane * 8;                              // cols % 8 == 0 and tn % 8 == 0: all 8 exist or none
+            return (j < nrows_w && ch < nch && c < ncols)
+                       ? __ldg(reinterpret_cast<const uint4 *>(wtile + (size_t)(i_begin + warp + j * (A1_THREADS / 32)) * g.cols + c))
+                       : make_uint4(0, 0, 0, 0);
+        };
+        uint32_t n_i = 0, n_a = 0, n_l = 0;
+        // groups of four chunks (1024 columns of a row): a warp keeps 2 KB requested ahead of what it evaluates
+        const int ngr = (nch + 3) >> 2;
+        uint4 wnext[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) wnext[u] = load_w(0, u);
+        for (int j = 0; j < nrows_w; ++j) {
+            const int i = i_begin + warp + j * (A1_THREADS / 32);
             const uint32_t *ipw = ip + ((size_t)tile * g.tm + i) * g.kw;
-            const uint16_t *wrow = W + (size_t)(tr * g.tm + i) * g.cols + (size_t)tc * g.tn;
-            for (int c0 = 0; c0 < ncols; c0 += 256) {                       // a lane owns 8 consecutive columns
-                const int c = c0 + lane * 8;
-                uint32_t bits = 0;                                          // index bits of the word that holds them
+            for (int gr4 = 0; gr4 < ngr; ++gr4) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) v[u] = wnext[u];
+                const int jn = gr4 + 1 < ngr ? j : j + 1, gn = gr4 + 1 < ngr ? gr4 + 1 : 0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) wnext[u] = load_w(jn, gn * 4 + u);
+                uint32_t bits[4] = {0u, 0u, 0u, 0u};                        // index bits of the words that hold this lane's columns
+                const int word0 = gr4 * 32 + (lane >> 2);                   // chunk u: word0 + 8 u
                 for (int lb = 0; lb < g.kw; ++lb) {
                     uint32_t x = __ldg(ipw + lb);                           // warp-uniform: no divergence below
                     if (lb == g.kw - 1) x &= tail;
                     while (x) {
-                        const int l = lb * 32 + __ffs(x) - 1;
+                        const uint32_t *pl = a1_planes + (lb * 32 + __ffs(x) - 1) * tnw;
                         x &= x - 1;
-                        if (c < ncols) bits |= a1_planes[l * tnw + (c >> 5)];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) bits[u] |= pl[min(word0 + 8 * u, tnw - 1)];
                     }
                 }
-                if (c < ncols) {                                            // cols % 8 == 0 and tn % 8 == 0: all 8 exist
-                    const uint4 v = *reinterpret_cast<const uint4 *>(wrow + c);
-                    const uint32_t by = bits >> (c & 31);
-                    const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-                    float cf = 0.f;
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        cost_element((e & 1) ? (ww[e >> 1] >> 16) : (ww[e >> 1] & 0xFFFFu), (by >> e) & 1u, theta, acc, cf);
-                    acc.cost += (double)cf;
+                for (int u = 0; u < 4; ++u) {
+                    const int c = (gr4 * 4 + u) * 256 + lane * 8;
+                    if (c < ncols) {
+                        float cf = 0.f;
+                        cost_chunk(v[u], bits[u] >> (c & 31), theta, n_i, n_a, n_l, cf);
+                        acc.cost += (double)cf;
+                    }
                 }
             }
         }
+        acc.kept_i = n_i; acc.kept_a = n_a; acc.lost = n_l;
     } else {
         // any shape: one column per lane, Eq. 3 evaluated per element from the packed words
         for (int i = i_begin + warp; i < i_end; i += A1_THREADS / 32) {
