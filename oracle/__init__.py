@@ -7,6 +7,7 @@ imports nothing from them.
 
 Functions (citations are to the paper):
   decode_mask          Eq. 3 applied tile by tile (Section 3.1).
+  decode_mask_ranks    the same with one rank per tile (Section 3.1, last paragraph).
   masked_gemm          Y = X (W .* Ia)^T with Ia as the masking layer (Sections 2, 2.2).
   masked_gemm_samples  the same two definitions evaluated only at chosen outputs.
   bf16_to_f64          exact widening of bf16 bit patterns.
@@ -50,6 +51,8 @@ def _load():
         i64, vp = ctypes.c_int64, ctypes.c_void_p
         lib.lrbi_oracle_decode.argtypes = [i64] * 5 + [vp] * 3
         lib.lrbi_oracle_decode.restype = None
+        lib.lrbi_oracle_decode_ranks.argtypes = [i64] * 5 + [vp] * 4
+        lib.lrbi_oracle_decode_ranks.restype = None
         lib.lrbi_oracle_masked_gemm.argtypes = [i64] * 3 + [vp] * 4
         lib.lrbi_oracle_masked_gemm.restype = None
         lib.lrbi_oracle_masked_gemm_samples.argtypes = [i64] * 5 + [vp] * 4 + [i64] + [vp] * 3
@@ -95,6 +98,25 @@ def decode_mask(Ip: np.ndarray, Iz: np.ndarray, rows: int, cols: int) -> np.ndar
         raise ValueError("factor entries must be 0 or 1")
     M = np.empty((rows, cols), dtype=np.uint8)
     _load().lrbi_oracle_decode(rows, cols, tm, tn, k, Ip.ctypes.data, Iz.ctypes.data, M.ctypes.data)
+    return M
+
+
+def decode_mask_ranks(Ip: np.ndarray, Iz: np.ndarray, ranks: np.ndarray, rows: int, cols: int) -> np.ndarray:
+    """Tiled Boolean product with one rank per tile: tile t uses Ip[..., :ranks[t]] and Iz[..., :ranks[t], :].
+
+    Ip: uint8 [GR, GC, tm, kmax], Iz: uint8 [GR, GC, kmax, tn], ranks: [GR*GC] (row-major grid order).
+    """
+    Ip = _c(Ip, np.uint8)
+    Iz = _c(Iz, np.uint8)
+    ranks = _c(ranks, np.int32).ravel()
+    GR, GC, tm, kmax = Ip.shape
+    tn = Iz.shape[3]
+    if Iz.shape[:3] != (GR, GC, kmax) or (GR, GC) != _grid(rows, cols, tm, tn) or ranks.size != GR * GC:
+        raise ValueError("factor shapes do not match the tile grid")
+    if ranks.min(initial=0) < 0 or ranks.max(initial=0) > kmax:
+        raise ValueError("a rank lies outside 0..kmax")
+    M = np.empty((rows, cols), dtype=np.uint8)
+    _load().lrbi_oracle_decode_ranks(rows, cols, tm, tn, kmax, ranks.ctypes.data, Ip.ctypes.data, Iz.ctypes.data, M.ctypes.data)
     return M
 
 

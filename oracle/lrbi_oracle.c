@@ -25,7 +25,7 @@
  * Threads (OpenMP) split the OUTER loop only; the arithmetic order inside one
  * output element never depends on the thread count.
  *
- * All four entry points are pinned by tests that do not use this file to make
+ * All entry points are pinned by tests that do not use this file to make
  * their expected values (the paper's printed worked example, brute-force
  * enumeration on tiny tiles, closed-form special cases, numpy's fp64 matmul for
  * the all-ones mask).  Nothing here is "parity unpinned".
@@ -70,6 +70,32 @@ void lrbi_oracle_decode(int64_t rows, int64_t cols, int64_t tm, int64_t tn, int6
             const uint8_t *ip_row = Ip + (tile * tm + i) * k;
             const uint8_t *iz_tile = Iz + tile * k * tn;
             M[r * cols + c] = boolean_dot(ip_row, iz_tile, k, tn, j);
+        }
+    }
+}
+
+/*
+ * The same product when every tile has its own rank (Section 3.1, last paragraph: each submatrix may
+ * choose a different rank).  The factors are stored with room for kmax = the largest rank,
+ *   Ip : [GR][GC][tm][kmax] bytes,  Iz : [GR][GC][kmax][tn] bytes,  ranks : [GR*GC],
+ * and tile t uses its first ranks[t] columns of Ip / rows of Iz only: whatever lies beyond is ignored.
+ */
+void lrbi_oracle_decode_ranks(int64_t rows, int64_t cols, int64_t tm, int64_t tn, int64_t kmax,
+                              const int32_t *ranks, const uint8_t *Ip, const uint8_t *Iz, uint8_t *M)
+{
+    const int64_t GC = (cols + tn - 1) / tn;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const int64_t tr = r / tm, i = r % tm;
+        for (int64_t c = 0; c < cols; ++c) {
+            const int64_t tc = c / tn, j = c % tn;
+            const int64_t tile = tr * GC + tc;
+            const uint8_t *ip_row = Ip + (tile * tm + i) * kmax;
+            const uint8_t *iz_tile = Iz + tile * kmax * tn;
+            uint8_t acc = 0;
+            for (int64_t l = 0; l < ranks[tile]; ++l)            /* Eq. 3 with k = the tile's own rank */
+                acc |= (uint8_t)(ip_row[l] & iz_tile[l * tn + j]);
+            M[r * cols + c] = acc;
         }
     }
 }

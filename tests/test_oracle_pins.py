@@ -285,3 +285,32 @@ def test_generator_is_seeded_and_shaped():
     # bf16 rounding: nearest, ties to even
     x = np.array([1.0, 1.00390625, 1.01171875, -1.00390625], dtype=np.float32)   # 1, 1+2^-8 (tie), 1+3*2^-8 (tie), ...
     assert synth.f32_to_bf16_bits(x).tolist() == [0x3F80, 0x3F80, 0x3F82, 0xBF80]
+
+
+# --------------------------------------------------------------------------- one rank per tile
+def test_decode_with_one_rank_per_tile():
+    """Section 3.1, last paragraph.  Pinned by what it must reduce to: every tile decoded on its own, untiled,
+    from the first ranks[t] columns/rows of its factors (OR of outer products); equal ranks give the plain
+    tiled decode; what lies beyond a tile's rank changes nothing; rank 0 gives an empty tile."""
+    rng = np.random.default_rng(21)
+    rows, cols, tm, tn, kmax = 11, 13, 4, 5, 6
+    gr, gc = -(-rows // tm), -(-cols // tn)
+    Ip = (rng.random((gr, gc, tm, kmax)) < 0.35).astype(np.uint8)
+    Iz = (rng.random((gr, gc, kmax, tn)) < 0.35).astype(np.uint8)
+    ranks = rng.integers(0, kmax + 1, gr * gc).astype(np.int32)
+    ranks[0], ranks[1] = 0, kmax
+    M = oracle.decode_mask_ranks(Ip, Iz, ranks, rows, cols)
+    for tr in range(gr):
+        for tc in range(gc):
+            k = ranks[tr * gc + tc]
+            want = or_of_outer_products(Ip[tr, tc][:, :k], Iz[tr, tc][:k, :]) if k else np.zeros((tm, tn), np.uint8)
+            blk = M[tr * tm:(tr + 1) * tm, tc * tn:(tc + 1) * tn]
+            assert (blk == want[:blk.shape[0], :blk.shape[1]]).all()
+    assert not M[:tm, :tn].any()                                           # rank 0
+    full = np.full(gr * gc, kmax, dtype=np.int32)
+    assert (oracle.decode_mask_ranks(Ip, Iz, full, rows, cols) == oracle.decode_mask(Ip, Iz, rows, cols)).all()
+    Ip2, Iz2 = Ip.copy(), Iz.copy()
+    for t in range(gr * gc):                                               # garbage beyond each tile's rank
+        Ip2.reshape(gr * gc, tm, kmax)[t][:, ranks[t]:] = 1
+        Iz2.reshape(gr * gc, kmax, tn)[t][ranks[t]:, :] = 1
+    assert (oracle.decode_mask_ranks(Ip2, Iz2, ranks, rows, cols) == M).all()
