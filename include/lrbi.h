@@ -231,6 +231,36 @@ LRBI_API lrbi_status lrbi_threshold_pack(const lrbi_layout *layout, const float 
 LRBI_API lrbi_status lrbi_index_cost(const lrbi_layout *layout, const uint16_t *W, float theta, const uint32_t *ip,
                                      const uint32_t *iz, lrbi_tile_cost *out, void *stream);
 
+/*
+ * Generalised layouts (Section 3.1, last paragraph: "each submatrix can optimally choose a different rank").
+ *
+ * Ranked layout: tile t (row-major grid order) has its own rank k_t, 0 <= k_t <= layout->rank (the layout's rank is
+ * then only the upper bound), and is packed with KW_t = ceil(k_t / 32) words per row of Ip / column of Iz:
+ *       ip[ip_offset[t] + i * KW_t + w],      iz[iz_offset[t] + j * KW_t + w]
+ * so a tile of low rank takes less room (k_t (tile_rows + tile_cols) bits, the index size of Section 2 for that
+ * tile).  A tile of rank 0 is empty: everything in it is pruned.  The three arrays are DEVICE arrays of GR*GC
+ * entries; offsets count 32-bit words.  Tile bases need only 4-byte alignment.
+ *   lrbi_decode_mask_ranked   Eq. 3 per tile with the tile's rank -> bit-packed mask (as lrbi_decode_mask)
+ *   lrbi_masked_gemm_ranked   the fused product (as lrbi_masked_gemm); the tensor-core kernel runs when the shape
+ *                             allows it (LRBI_ALGO_TENSOR's conditions), else a one-thread-per-output kernel
+ *
+ * lrbi_decode_mask_batch: the indices of n layers decoded by ONE launch per 32 layers (many small layers, e.g. the
+ * blocks of a network, cost one launch latency instead of n).  layouts, ip, iz, mask_out are HOST arrays of n
+ * entries; the pointers they hold are device pointers as for lrbi_decode_mask.
+ */
+typedef struct {
+    const int32_t *ranks;     /* device, [GR*GC]                                   */
+    const int64_t *ip_offset; /* device, [GR*GC], first word of tile t in ip       */
+    const int64_t *iz_offset; /* device, [GR*GC], first word of tile t in iz       */
+} lrbi_tile_ranks;
+LRBI_API lrbi_status lrbi_decode_mask_ranked(const lrbi_layout *layout, const lrbi_tile_ranks *ranks, const uint32_t *ip,
+                                             const uint32_t *iz, uint32_t *mask_out, void *stream);
+LRBI_API lrbi_status lrbi_masked_gemm_ranked(const lrbi_layout *layout, const lrbi_tile_ranks *ranks, const uint16_t *W,
+                                             const uint32_t *ip, const uint32_t *iz, const uint16_t *X, int32_t batch,
+                                             void *Y, int32_t y_dtype, int32_t algo, void *stream);
+LRBI_API lrbi_status lrbi_decode_mask_batch(int32_t n, const lrbi_layout *layouts, const uint32_t *const *ip,
+                                            const uint32_t *const *iz, uint32_t *const *mask_out, void *stream);
+
 /* Which kernel LRBI_ALGO_AUTO would run for this layout and batch (an LRBI_ALGO_* value). */
 LRBI_API int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batch);
 

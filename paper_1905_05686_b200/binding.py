@@ -38,6 +38,11 @@ class GemmPlan(ctypes.Structure):
                 ("scratch_bytes", ctypes.c_uint64)]
 
 
+class TileRanks(ctypes.Structure):
+    """lrbi_tile_ranks: device arrays with one rank and two word offsets per tile."""
+    _fields_ = [("ranks", ctypes.c_void_p), ("ip_offset", ctypes.c_void_p), ("iz_offset", ctypes.c_void_p)]
+
+
 class Layout(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int32), ("cols", ctypes.c_int32), ("tile_rows", ctypes.c_int32),
                 ("tile_cols", ctypes.c_int32), ("rank", ctypes.c_int32)]
@@ -92,6 +97,12 @@ def lib():
         L.lrbi_threshold_pack.restype = i32
         L.lrbi_index_cost.argtypes = [lp, vp, ctypes.c_float, vp, vp, vp, vp]
         L.lrbi_index_cost.restype = i32
+        L.lrbi_decode_mask_ranked.argtypes = [lp, ctypes.POINTER(TileRanks), vp, vp, vp, vp]
+        L.lrbi_decode_mask_ranked.restype = i32
+        L.lrbi_masked_gemm_ranked.argtypes = [lp, ctypes.POINTER(TileRanks), vp, vp, vp, vp, i32, vp, i32, i32, vp]
+        L.lrbi_masked_gemm_ranked.restype = i32
+        L.lrbi_decode_mask_batch.argtypes = [i32, lp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
+        L.lrbi_decode_mask_batch.restype = i32
         L.lrbi_launch_count.argtypes = []
         L.lrbi_launch_count.restype = ctypes.c_uint64
         L.lrbi_device_status.argtypes = [i32]
@@ -175,6 +186,59 @@ def lrbi_decode_mask(layer, ip: torch.Tensor, iz: torch.Tensor, mask_out: torch.
     if rc != OK:
         raise LrbiError(rc, "lrbi_decode_mask")
     return mask_out
+
+
+def _tile_ranks(lay, ranks, ip_off, iz_off):
+    tiles = (-(-lay.rows // lay.tile_rows)) * (-(-lay.cols // lay.tile_cols))
+    if ranks.numel() != tiles or ip_off.numel() != tiles or iz_off.numel() != tiles:
+        raise ValueError("one rank and one pair of offsets per tile")
+    return TileRanks(_dev(ranks, torch.int32, "ranks").value, _dev(ip_off, torch.int64, "ip_offset").value,
+                     _dev(iz_off, torch.int64, "iz_offset").value)
+
+
+def lrbi_decode_mask_ranked(layer, ranks, ip_off, iz_off, ip, iz, mask_out=None, stream=None) -> torch.Tensor:
+    """lrbi_decode_mask for a ranked layout (one rank per tile; `layer.rank` is the upper bound)."""
+    lay = Layout.of(layer)
+    tr = _tile_ranks(lay, ranks, ip_off, iz_off)
+    if mask_out is None:
+        mask_out = torch.empty((lay.rows, (lay.cols + 31) // 32), dtype=torch.int32, device=ip.device)
+    rc = lib().lrbi_decode_mask_ranked(ctypes.byref(lay), ctypes.byref(tr), _dev(ip, torch.int32, "ip"), _dev(iz, torch.int32, "iz"),
+                                       _dev(mask_out, torch.int32, "mask_out"), _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_decode_mask_ranked")
+    return mask_out
+
+
+def lrbi_masked_gemm_ranked(layer, ranks, ip_off, iz_off, W, ip, iz, X, Y=None, y_dtype=torch.bfloat16, algo=ALGO_AUTO,
+                            stream=None) -> torch.Tensor:
+    """lrbi_masked_gemm for a ranked layout."""
+    lay = Layout.of(layer)
+    tr = _tile_ranks(lay, ranks, ip_off, iz_off)
+    if tuple(W.shape) != (lay.rows, lay.cols) or X.dim() != 2 or X.shape[1] != lay.cols:
+        raise ValueError("W / X shapes do not match the layout")
+    batch = X.shape[0]
+    if Y is None:
+        Y = torch.empty((batch, lay.rows), dtype=y_dtype, device=X.device)
+    elif tuple(Y.shape) != (batch, lay.rows) or Y.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("Y has the wrong shape or dtype")
+    rc = lib().lrbi_masked_gemm_ranked(ctypes.byref(lay), ctypes.byref(tr), _dev(W, torch.bfloat16, "W"), _dev(ip, torch.int32, "ip"),
+                                       _dev(iz, torch.int32, "iz"), _dev(X, torch.bfloat16, "X"), batch, _dev(Y, Y.dtype, "Y"),
+                                       Y_F32 if Y.dtype == torch.float32 else Y_BF16, algo, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_masked_gemm_ranked")
+    return Y
+
+
+def lrbi_decode_mask_batch(layers, ips, izs, stream=None):
+    """Decode the indices of several layers with one launch per 32 layers; returns the list of masks."""
+    n = len(layers)
+    lays = (Layout * n)(*[Layout.of(l) for l in layers])
+    masks = [torch.empty((l.rows, (l.cols + 31) // 32), dtype=torch.int32, device=ips[0].device) for l in lays]
+    arr = lambda ts, what: (ctypes.c_void_p * n)(*[_dev(t, torch.int32, what).value for t in ts])
+    rc = lib().lrbi_decode_mask_batch(n, lays, arr(ips, "ip"), arr(izs, "iz"), arr(masks, "mask_out"), _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_decode_mask_batch")
+    return masks
 
 
 def lrbi_threshold_pack(layer, mp: torch.Tensor, mz: torch.Tensor, tp: torch.Tensor, tz: torch.Tensor, stream=None):

@@ -191,6 +191,59 @@ lrbi_status lrbi_index_cost(const lrbi_layout *layout, const uint16_t *W, float 
     return launch_index_cost(make_geo(*layout), W, theta, ip, iz, out, static_cast<cudaStream_t>(stream));
 }
 
+static bool ranks_ok(const lrbi_tile_ranks *r) { return r && r->ranks && r->ip_offset && r->iz_offset; }
+static TileRanks to_ranks(const lrbi_tile_ranks *r)
+{
+    TileRanks t = {r->ranks, reinterpret_cast<const long long *>(r->ip_offset), reinterpret_cast<const long long *>(r->iz_offset)};
+    return t;
+}
+
+lrbi_status lrbi_decode_mask_ranked(const lrbi_layout *layout, const lrbi_tile_ranks *ranks, const uint32_t *ip,
+                                    const uint32_t *iz, uint32_t *mask_out, void *stream)
+{
+    if (!layout_ok(layout) || !ranks_ok(ranks) || !ip || !iz || !mask_out || !aligned16(mask_out)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    return launch_decode_ranked(make_geo(*layout), to_ranks(ranks), ip, iz, mask_out, static_cast<cudaStream_t>(stream));
+}
+
+lrbi_status lrbi_masked_gemm_ranked(const lrbi_layout *layout, const lrbi_tile_ranks *ranks, const uint16_t *W,
+                                    const uint32_t *ip, const uint32_t *iz, const uint16_t *X, int32_t batch, void *Y,
+                                    int32_t y_dtype, int32_t algo, void *stream)
+{
+    if (!layout_ok(layout) || !ranks_ok(ranks) || !W || !ip || !iz || !X || !Y || batch < 1) return LRBI_ERR_INVALID_ARG;
+    if (y_dtype != LRBI_Y_BF16 && y_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(X) || !aligned16(Y)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    const Geo g = make_geo(*layout);
+    const TileRanks rk = to_ranks(ranks);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (algo == LRBI_ALGO_AUTO) algo = gemm_tc_supported(g, batch) ? LRBI_ALGO_TENSOR : LRBI_ALGO_GENERIC;
+    switch (algo) {
+    case LRBI_ALGO_GENERIC: return launch_gemm_ranked_generic(g, rk, W, ip, iz, X, batch, Y, y_dtype, s);
+    case LRBI_ALGO_TENSOR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 0, &rk);
+    case LRBI_ALGO_TENSOR_PAIR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 1, &rk);
+    case LRBI_ALGO_TENSOR_PAIR2: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 2, &rk);
+    default: return LRBI_ERR_INVALID_ARG;
+    }
+}
+
+lrbi_status lrbi_decode_mask_batch(int32_t n, const lrbi_layout *layouts, const uint32_t *const *ip,
+                                   const uint32_t *const *iz, uint32_t *const *mask_out, void *stream)
+{
+    if (n < 1 || n > 4096 || !layouts || !ip || !iz || !mask_out) return LRBI_ERR_INVALID_ARG;
+    Geo *g = new (std::nothrow) Geo[n];
+    if (!g) return LRBI_ERR_CUDA;
+    lrbi_status st = LRBI_OK;
+    for (int l = 0; l < n && st == LRBI_OK; ++l) {
+        if (!layout_ok(&layouts[l]) || !ip[l] || !iz[l] || !mask_out[l] || !aligned16(mask_out[l])) st = LRBI_ERR_INVALID_ARG;
+        else g[l] = make_geo(layouts[l]);
+    }
+    if (st == LRBI_OK && device_timeout_seen()) st = LRBI_ERR_TIMEOUT;
+    if (st == LRBI_OK) st = launch_decode_batch(n, g, ip, iz, mask_out, static_cast<cudaStream_t>(stream));
+    delete[] g;
+    return st;
+}
+
 uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t lrbi_device_status(int32_t clear)

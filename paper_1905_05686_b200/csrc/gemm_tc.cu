@@ -156,27 +156,51 @@ __device__ __forceinline__ void cp_async_16(void *dst_smem, const void *src, int
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
+// Rank and words per row/column of the tile that holds rows o0.. and columns c0.. (one rank per tile when `rk`
+// carries arrays, else the layout's rank), and the first factor words of that tile.
+__device__ __forceinline__ void panel_tile(const Geo &g, const TileRanks &rk, const uint32_t *ip, const uint32_t *iz,
+                                           int c0, int o0, int &k, int &kw, const uint32_t *&ipt, const uint32_t *&izt)
+{
+    const int tr = min(o0, g.rows - 1) / g.tm, tc = min(c0, g.cols - 1) / g.tn;
+    const size_t tile = (size_t)tr * g.gc + tc;
+    if (rk.ranks) {
+        k = __ldg(rk.ranks + tile);
+        kw = (k + 31) >> 5;
+        ipt = ip + __ldg(rk.ip_offset + tile);
+        izt = iz + __ldg(rk.iz_offset + tile);
+    } else {
+        k = g.k;
+        kw = g.kw;
+        ipt = ip + tile * g.tm * g.kw;
+        izt = iz + tile * g.tn * g.kw;
+    }
+}
+
 // Stage the factor words of one panel: the Iz words of its `pw32` columns (first column c0, tile row tr)
-// and the Ip words of the block's 128 rows (first row o0).  Words outside the tile are written as zero.
+// and the Ip words of the block's 128 rows (first row o0), kw words each (the rank of the panel's tile).
+// Words outside the tile are written as zero.
 // Asynchronous copies (one commit group); the caller waits for them.  dt = 0 .. nthreads-1.
-__device__ __forceinline__ void stage_panel_factors(const Geo &g, const uint32_t *__restrict__ ip,
+__device__ __forceinline__ void stage_panel_factors(const Geo &g, const TileRanks &rk, const uint32_t *__restrict__ ip,
                                                     const uint32_t *__restrict__ iz, uint32_t *iz_stage,
                                                     uint32_t *ip_stage, int pw32, int c0, int o0, int dt, int nthreads)
 {
-    const int zwords = pw32 * g.kw, xwords = TC_BM * g.kw;
+    int k, kw;
+    const uint32_t *ipt, *izt;
+    panel_tile(g, rk, ip, iz, c0, o0, k, kw, ipt, izt);
+    const int zwords = pw32 * kw, xwords = TC_BM * kw;
     if (o0 >= g.rows) {                                  // a block without rows of W (second CTA of a ragged pair)
         for (int q = dt; q < zwords; q += nthreads) iz_stage[q] = 0u;
         for (int q = dt; q < xwords; q += nthreads) ip_stage[q] = 0u;
+        cp_async_commit();
         return;
     }
-    // 16-byte copies need 16-byte aligned sources: tile bases are, unless a tile holds an odd word count
-    const bool z_vec = ((g.tn * g.kw) & 3) == 0, x_vec = ((g.tm * g.kw) & 3) == 0;
-    const int tr = o0 / g.tm, i0 = o0 - tr * g.tm;       // tile row, first row of the block inside its tile
-    const int tc = c0 / g.tn, j0 = c0 - tc * g.tn;       // tile column, first column of the panel inside its tile
-    const size_t tile = (size_t)tr * g.gc + tc;
-    const uint32_t *zsrc = iz + (tile * g.tn + j0) * g.kw;
-    const uint32_t *xsrc = ip + (tile * g.tm + i0) * g.kw;
-    const int zvalid = (g.tn - j0) * g.kw, xvalid = (g.tm - i0) * g.kw;   // words that exist in the tile
+    const int i0 = o0 - (o0 / g.tm) * g.tm;              // first row of the block inside its tile
+    const int j0 = c0 - (c0 / g.tn) * g.tn;              // first column of the panel inside its tile
+    const uint32_t *zsrc = izt + (size_t)j0 * kw;
+    const uint32_t *xsrc = ipt + (size_t)i0 * kw;
+    // 16-byte copies need 16-byte aligned sources (tile bases of a ranked layout need not be)
+    const bool z_vec = (reinterpret_cast<uintptr_t>(zsrc) & 15u) == 0, x_vec = (reinterpret_cast<uintptr_t>(xsrc) & 15u) == 0;
+    const int zvalid = (g.tn - j0) * kw, xvalid = (g.tm - i0) * kw;   // words that exist in the tile
     for (int q = dt * 4; q < zwords; q += nthreads * 4) {
         const int n = min(4, max(0, zvalid - q));
         if (z_vec) cp_async_16(iz_stage + q, zsrc + (n > 0 ? q : 0), n * 4);
@@ -249,7 +273,7 @@ __device__ __forceinline__ int warp_of_thread_decoder_group(unsigned tid)
 // one block's epilogue and panel hand-overs overlap the other's MMAs.
 template <int BN, int PW, bool PAIR>
 __global__ void __launch_bounds__(tc_threads(BN), BN > 256 ? 1 : 2)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g, TileRanks rk,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
                int stages, int *status)
@@ -299,7 +323,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     // Long-latency requests first: the decoder warps ask for the factor words of their first panel, one
     // thread warms the TMA descriptors; both overlap the barrier and tensor-memory set-up below.
     if (warp >= 2 + TC_MASK_WARPS && dgrp * KBP < nkb)   // group g starts with panel g
-        stage_panel_factors(g, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + dgrp * KBP) * TC_BK, o0,
+        stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + dgrp * KBP) * TC_BK, o0,
                             (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1), TC_DECODE_WARPS * 32);
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
@@ -406,17 +430,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         // ------------------------------------------------------------- index decoders
         const int dt = (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1);   // 0..127: row of the block this thread decodes
         const int dw = dt >> 5;                         // decoder warp 0..3
-        const uint32_t tail = tail_mask(g.k);
         const int tr = o0 / g.tm;                       // the 128 rows lie in one tile row
         const int i0 = o0 - tr * g.tm;                  // first row of the block inside its tile
         const bool row_ok = o0 + dt < g.rows && i0 + dt < g.tm;
         const int bit_col = column_of_bit(lane);        // column (0..31) this lane stands for in a transpose
-        const int npairs = g.kw * PW;                   // (32-plane block, index word) pairs of a panel
         const int npanels = (nkb + KBP - 1) / KBP;
 
         auto stage_factors = [&](int P) {
             if (P < npanels)
-                stage_panel_factors(g, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + P * KBP) * TC_BK, o0, dt, TC_DECODE_WARPS * 32);
+                stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + P * KBP) * TC_BK, o0, dt, TC_DECODE_WARPS * 32);
         };
 
         uint32_t dsync_parity = 0;
@@ -433,6 +455,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             const int buf = P & 1;
             uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
             const int c0 = (kb_begin + P * KBP) * TC_BK;
+            // rank of the panel's tile (the layout's, or the tile's own in a ranked layout)
+            int kp = g.k, kwp = g.kw;
+            if (rk.ranks) {
+                kp = __ldg(rk.ranks + (size_t)min(tr, g.gr - 1) * g.gc + min(c0, g.cols - 1) / g.tn);
+                kwp = (kp + 31) >> 5;
+            }
+            const uint32_t tail = tail_mask(kp);
+            const int npairs = kwp * PW;                 // (32-plane block, index word) pairs of the panel
             cp_async_wait_all();                         // this thread's copies for panel P have landed
             dsync();                                     // ... and everybody else's
             if (!ok) break;
@@ -444,8 +474,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 for (int t = 0; t < 4; ++t) {
                     const int pi = dw + TC_DECODE_WARPS * (n0 + t);
                     const int lb = pi / PW, col = (pi % PW) * 32 + bit_col;
-                    z[t] = (pi < npairs && c0 + col < g.cols) ? iz_stage[col * g.kw + lb] : 0u;
-                    if (lb == g.kw - 1) z[t] &= tail;
+                    z[t] = (pi < npairs && c0 + col < g.cols) ? iz_stage[col * kwp + lb] : 0u;
+                    if (lb == kwp - 1) z[t] &= tail;
                 }
                 warp_transpose32_x4(z, lane);
 #pragma unroll
@@ -458,8 +488,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             uint32_t xw[8];
 #pragma unroll
             for (int lb = 0; lb < 8; ++lb) {
-                xw[lb] = (row_ok && lb < g.kw) ? ip_stage[dt * g.kw + lb] : 0u;
-                if (lb == g.kw - 1) xw[lb] &= tail;
+                xw[lb] = (row_ok && lb < kwp) ? ip_stage[dt * kwp + lb] : 0u;
+                if (lb == kwp - 1) xw[lb] &= tail;
             }
             dsync();                                     // planes complete, factor staging consumed
             if (!ok) break;
@@ -805,7 +835,7 @@ static int device_sm_count(int *dev_out)
 template <int BN, int PW, bool PAIR>
 static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const uint16_t *W, const uint32_t *ip,
                              const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype,
-                             cudaStream_t s, float *partials)
+                             cudaStream_t s, float *partials, const TileRanks &rk)
 {
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) { note_cuda_error(-1); return LRBI_ERR_CUDA; }
@@ -852,7 +882,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int *status = device_status_ptr();
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, ip, iz, batch, Y, y_dtype, partials, plan.kb_per_split, plan.stages, status);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, rk, ip, iz, batch, Y, y_dtype, partials, plan.kb_per_split, plan.stages, status);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
@@ -869,8 +899,9 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
 // `fixed_scratch` != nullptr: the caller forbids allocation, partial sums go there (fixed_bytes) or nowhere.
 static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s,
-                          float *fixed_scratch, size_t fixed_bytes, int force = 0)
+                          float *fixed_scratch, size_t fixed_bytes, int force = 0, const TileRanks *ranks = nullptr)
 {
+    const TileRanks rk = ranks ? *ranks : TileRanks{nullptr, nullptr, nullptr};
     if (!gemm_tc_supported(g, batch)) return LRBI_ERR_UNSUPPORTED;    // shape errors come before device errors
     int dev = -1;
     const int sm_count = device_sm_count(&dev);
@@ -886,7 +917,7 @@ static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, c
     }
 #define LRBI_TC_CASE(BN_, PW_, PAIR_) \
     if (plan.bn == BN_ && plan.pw == PW_ && plan.pair == PAIR_) \
-        return launch_tc<BN_, PW_, PAIR_>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials);
+        return launch_tc<BN_, PW_, PAIR_>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials, rk);
     LRBI_TC_CASE(16, 8, false) LRBI_TC_CASE(16, 2, false)
     LRBI_TC_CASE(32, 8, false) LRBI_TC_CASE(32, 2, false)
     LRBI_TC_CASE(64, 8, false) LRBI_TC_CASE(64, 2, false)
@@ -898,9 +929,9 @@ static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, c
 }
 
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force)
+                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force, const TileRanks *ranks)
 {
-    return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, nullptr, 0, force);
+    return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, nullptr, 0, force, ranks);
 }
 
 bool gemm_tc_plan(const Geo &g, int batch, int force, lrbi_gemm_plan *out)

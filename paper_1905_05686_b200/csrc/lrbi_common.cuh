@@ -29,6 +29,13 @@ inline Geo make_geo(const lrbi_layout &l)
     return g;
 }
 
+// One rank per tile (null pointers: the layout's rank for every tile).  Offsets count 32-bit words.
+struct TileRanks {
+    const int32_t *ranks;
+    const long long *ip_offset;
+    const long long *iz_offset;
+};
+
 // Codes a kernel leaves in the device status word when a bounded wait runs out.
 enum : int {
     DEV_OK = 0,
@@ -129,7 +136,8 @@ bool gemm_tc_supported(const Geo &g, int batch);
 // When it splits K the launcher keeps fp32 partial sums in the library-owned buffer of the device.
 // force: 0 = instantiation chosen by shape, 1 = CTA pairs (one accumulator), 2 = CTA pairs (two accumulators)
 lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
-                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force = 0);
+                           const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force = 0,
+                           const TileRanks *ranks = nullptr);   // ranks: one rank per tile (a ranked layout), or null
 
 // Variant that keeps K-split partial sums in the library's fixed device array; allocates nothing.
 lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,
@@ -138,6 +146,14 @@ size_t gemm_tc_scratch_bytes(const Geo &g, int batch);   // fp32 partial sums th
 lrbi_status launch_bounded_wait_selftest(unsigned limit_us, cudaStream_t s);
 bool gemm_tc_plan(const Geo &g, int batch, int force, lrbi_gemm_plan *out);   // fills the tensor-core fields of the plan
 
+
+// Generalised layouts: one rank per tile, several layers per launch.
+lrbi_status launch_decode_ranked(const Geo &g, const TileRanks &rk, const uint32_t *ip, const uint32_t *iz,
+                                 uint32_t *mask, cudaStream_t s);
+lrbi_status launch_decode_batch(int n, const Geo *g, const uint32_t *const *ip, const uint32_t *const *iz,
+                                uint32_t *const *mask, cudaStream_t s);
+lrbi_status launch_gemm_ranked_generic(const Geo &g, const TileRanks &rk, const uint16_t *W, const uint32_t *ip,
+                                       const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
 
 // Inner loop of Algorithm 1.
 lrbi_status launch_threshold_pack(const Geo &g, const float *mp, const float *mz, const float *tp, const float *tz,

@@ -139,6 +139,31 @@ def pack_iz(Iz: np.ndarray) -> np.ndarray:
     return _pack_last_axis(np.swapaxes(Iz, 2, 3)).reshape(-1).copy()
 
 
+def pack_ranked(Ip: np.ndarray, Iz: np.ndarray, ranks: np.ndarray):
+    """Ranked layout: tile t keeps its first ranks[t] bits, packed with ceil(ranks[t] / 32) words per row / column,
+    tiles one after the other.  Returns (ip_words, iz_words, ip_offset, iz_offset), offsets in words (int64)."""
+    gr, gc, tm, kmax = Ip.shape
+    tn = Iz.shape[3]
+    ranks = np.asarray(ranks, dtype=np.int64).ravel()
+    ipw, izw, ipo, izo = [], [], [], []
+    n_ip = n_iz = 0
+    for t in range(gr * gc):
+        k = int(ranks[t])
+        ipo.append(n_ip)
+        izo.append(n_iz)
+        if k:
+            a = _pack_last_axis(Ip.reshape(gr * gc, tm, kmax)[t][:, :k]).reshape(-1)
+            z = _pack_last_axis(np.swapaxes(Iz.reshape(gr * gc, kmax, tn)[t][:k, :], 0, 1)).reshape(-1)
+            ipw.append(a)
+            izw.append(z)
+            n_ip += a.size
+            n_iz += z.size
+    cat = lambda parts: np.concatenate(parts).astype(np.uint32) if parts else np.zeros(0, dtype=np.uint32)
+    # keep the arrays non-empty and padded to whole 16-byte vectors
+    pad = lambda a: np.concatenate([a, np.zeros((-a.size) % 4 + (4 if a.size == 0 else 0), dtype=np.uint32)])
+    return pad(cat(ipw)), pad(cat(izw)), np.array(ipo, dtype=np.int64), np.array(izo, dtype=np.int64)
+
+
 def pack_mask(M: np.ndarray) -> np.ndarray:
     """[rows, cols] bytes -> uint32 [rows, ceil(cols/32)]; bit (c % 32) of word c // 32 = M[r, c]."""
     return _pack_last_axis(M)
