@@ -30,7 +30,18 @@ DEFAULT_WORKLOAD = "ffn_16384x4096"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu capture
 # summarised under profiles/ (null for workloads without a capture of the current kernel)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("ffn_16384x4096", 4096): 406_000_000,      # 290 MB read + 116 MB written (profiles/ncu_traffic_all_workloads.md)
+    ("lenet_fc1", 32): 1_050_000,
+    ("decode_4096", 0): 534_000,                # the 2 MiB mask is still in L2 when the kernel ends
+    ("decode_32768", 0): 104_200_000,
+    ("alexnet_fc", 1): 76_200_000,
+    ("alexnet_fc", 16): 78_900_000,             # both launches (K-split kernel + reduction)
+    ("alexnet_fc", 128): 97_500_000,
+    ("conv3x3_256", 12544): 59_100_000,         # Y (6.4 MB) is still in L2 when the kernel ends
+    ("alexnet_fc", -1): 76_200_000,
+    ("ffn_16384x4096", -1): 135_500_000,
+}
 # The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
 # batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
 OTHER_WORKLOADS = [("lenet_fc1", 32), ("decode_4096", 0), ("decode_32768", 0), ("alexnet_fc", 1), ("alexnet_fc", 16),
