@@ -10,6 +10,7 @@ Functions (citations are to the paper):
   decode_mask_ranks    the same with one rank per tile (Section 3.1, last paragraph).
   masked_gemm          Y = X (W .* Ia)^T with Ia as the masking layer (Sections 2, 2.2).
   masked_gemm_samples  the same two definitions evaluated only at chosen outputs.
+  masked_backward      dX = dY (W .* Ia), dW = (dY^T X) .* Ia: gradients of the masked layer (Section 2.2).
   bf16_to_f64          exact widening of bf16 bit patterns.
 Inner loop of Algorithm 1 (Section 2.1), in lrbi_alg1_oracle.c and, for the search itself, below:
   threshold            binary conversion of NMF factors, entry = 1 iff value >= T (sentence under Eq. 4).
@@ -55,6 +56,8 @@ def _load():
         lib.lrbi_oracle_decode_ranks.restype = None
         lib.lrbi_oracle_masked_gemm.argtypes = [i64] * 3 + [vp] * 4
         lib.lrbi_oracle_masked_gemm.restype = None
+        lib.lrbi_oracle_masked_backward.argtypes = [i64] * 3 + [vp] * 6
+        lib.lrbi_oracle_masked_backward.restype = None
         lib.lrbi_oracle_masked_gemm_samples.argtypes = [i64] * 5 + [vp] * 4 + [i64] + [vp] * 3
         lib.lrbi_oracle_masked_gemm_samples.restype = None
         lib.lrbi_oracle_bf16_to_f64.argtypes = [i64, vp, vp]
@@ -135,6 +138,20 @@ def masked_gemm(W_bits: np.ndarray, M: np.ndarray, X_bits: np.ndarray) -> np.nda
     Y = np.empty((B, N), dtype=np.float64)
     _load().lrbi_oracle_masked_gemm(B, N, K, W_bits.ctypes.data, M.ctypes.data, X_bits.ctypes.data, Y.ctypes.data)
     return Y
+
+
+def masked_backward(W_bits: np.ndarray, M: np.ndarray, X_bits: np.ndarray, dY_bits: np.ndarray):
+    """Gradients of Y = X (W .* M)^T for dY = dL/dY, in fp64: (dX [B, K], dW [N, K]); dW is zero where M is."""
+    W_bits, X_bits, dY_bits, M = _c(W_bits, np.uint16), _c(X_bits, np.uint16), _c(dY_bits, np.uint16), _c(M, np.uint8)
+    N, K = W_bits.shape
+    B = X_bits.shape[0]
+    if X_bits.shape != (B, K) or dY_bits.shape != (B, N) or M.shape != (N, K):
+        raise ValueError("shape mismatch")
+    dX = np.empty((B, K), dtype=np.float64)
+    dW = np.empty((N, K), dtype=np.float64)
+    _load().lrbi_oracle_masked_backward(B, N, K, W_bits.ctypes.data, M.ctypes.data, X_bits.ctypes.data, dY_bits.ctypes.data,
+                                        dX.ctypes.data, dW.ctypes.data)
+    return dX, dW
 
 
 def masked_gemm_samples(W_bits, Ip, Iz, X_bits, b_idx, o_idx) -> np.ndarray:

@@ -122,6 +122,37 @@ void lrbi_oracle_masked_gemm(int64_t B, int64_t N, int64_t K,
 }
 
 /*
+ * Backward pass of the masked layer (Section 2.2: the pruned network is retrained with the index Ia as its
+ * masking layer, so gradients flow through kept weights only).  With Y = X (W .* Ia)^T and dY = dL/dY:
+ *   dX[b][i] = sum_o  Ia[o][i] ? dY[b][o] * W[o][i] : nothing
+ *   dW[o][i] = Ia[o][i] ? sum_b dY[b][o] * X[b][i] : 0          (a pruned weight gets no gradient)
+ *   W : [N][K], M : [N][K] bytes, X : [B][K], dY : [B][N] (bf16 bits);  dX : [B][K], dW : [N][K] fp64.
+ */
+void lrbi_oracle_masked_backward(int64_t B, int64_t N, int64_t K, const uint16_t *W, const uint8_t *M,
+                                 const uint16_t *X, const uint16_t *dY, double *dX, double *dW)
+{
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t b = 0; b < B; ++b) {
+        for (int64_t i = 0; i < K; ++i) {
+            double s = 0.0;
+            for (int64_t o = 0; o < N; ++o)
+                if (M[o * K + i]) s += bf16_bits_to_double(dY[b * N + o]) * bf16_bits_to_double(W[o * K + i]);
+            dX[b * K + i] = s;
+        }
+    }
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t o = 0; o < N; ++o) {
+        for (int64_t i = 0; i < K; ++i) {
+            double s = 0.0;
+            if (M[o * K + i])
+                for (int64_t b = 0; b < B; ++b)
+                    s += bf16_bits_to_double(dY[b * N + o]) * bf16_bits_to_double(X[b * K + i]);
+            dW[o * K + i] = s;
+        }
+    }
+}
+
+/*
  * The same two definitions restricted to chosen outputs, for layers too large to
  * evaluate in full: for sample s the mask row o = o_idx[s] is decoded from its
  * tiles' factors (Eq. 3), then Y[b_idx[s]][o] is summed as above.

@@ -314,3 +314,28 @@ def test_decode_with_one_rank_per_tile():
         Ip2.reshape(gr * gc, tm, kmax)[t][:, ranks[t]:] = 1
         Iz2.reshape(gr * gc, kmax, tn)[t][ranks[t]:, :] = 1
     assert (oracle.decode_mask_ranks(Ip2, Iz2, ranks, rows, cols) == M).all()
+
+
+# --------------------------------------------------------------------------- masked backward
+def test_masked_backward():
+    """Pinned by numpy's fp64 matmul on the masked weights, by the adjoint identities that tie it to the (separately
+    pinned) forward product, and by the special masks: full mask = the plain GEMM gradients, empty mask = zeros."""
+    rng = np.random.default_rng(9)
+    B, N, K = 5, 7, 11
+    bits = lambda a: synth.f32_to_bf16_bits(a.astype(np.float32))
+    Wb, Xb, dYb = bits(rng.standard_normal((N, K))), bits(rng.standard_normal((B, K))), bits(rng.standard_normal((B, N)))
+    f = lambda b: synth.bf16_bits_to_f32(b).astype(np.float64)
+    for M in (np.ones((N, K), np.uint8), np.zeros((N, K), np.uint8), (rng.random((N, K)) < 0.4).astype(np.uint8)):
+        dX, dW = oracle.masked_backward(Wb, M, Xb, dYb)
+        assert np.allclose(dX, f(dYb) @ (f(Wb) * M), rtol=1e-12, atol=1e-12)       # [B,N] x [N,K]
+        assert np.allclose(dW, (f(dYb).T @ f(Xb)) * M, rtol=1e-12, atol=1e-12)     # ([N,B] x [B,K]) .* M
+        assert not dW[M == 0].any()
+        # <dY, Y(E)> = <dX, E> for any activations E, and <dY, Y with weights F> = <dW, F> for any weights F
+        Eb, Fb = bits(rng.standard_normal((B, K))), bits(rng.standard_normal((N, K)))
+        assert np.sum(f(dYb) * oracle.masked_gemm(Wb, M, Eb)) == pytest.approx(np.sum(dX * f(Eb)), rel=1e-10, abs=1e-10)
+        assert np.sum(f(dYb) * oracle.masked_gemm(Fb, M, Xb)) == pytest.approx(np.sum(dW * f(Fb)), rel=1e-10, abs=1e-10)
+    # a transposed operand would fail the shapes above (B, N, K all differ); a NaN in a pruned weight reaches neither
+    M = (rng.random((N, K)) < 0.5).astype(np.uint8)
+    Wn = Wb.copy()
+    Wn[M == 0] = 0x7FC0
+    assert np.array_equal(oracle.masked_backward(Wn, M, Xb, dYb)[0], oracle.masked_backward(Wb, M, Xb, dYb)[0])
