@@ -261,6 +261,32 @@ LRBI_API lrbi_status lrbi_masked_gemm_ranked(const lrbi_layout *layout, const lr
 LRBI_API lrbi_status lrbi_decode_mask_batch(int32_t n, const lrbi_layout *layouts, const uint32_t *const *ip,
                                             const uint32_t *const *iz, uint32_t *const *mask_out, void *stream);
 
+/*
+ * Backward pass of the masked layer (Section 2.2: the pruned network is retrained "using a masking layer" Ia, so
+ * gradients flow through kept weights only).  With Y = X (W .* Ia)^T and dY = dL/dY [batch][rows]:
+ *       dX[b][i] = sum_o  Ia[o][i] ? dY[b][o] * W[o][i] : 0          dW[o][i] = Ia[o][i] ? sum_b dY[b][o] * X[b][i] : 0
+ * fp32 accumulation; outputs bf16 (round to nearest even) or fp32 as the dtype argument says (LRBI_Y_*).
+ *
+ * lrbi_masked_gemm_dx   needs the weights TRANSPOSED: Wt [cols][rows] bf16 (keep that copy beside W and refresh it with
+ *       lrbi_transpose_bf16 when W changes).  It is the forward product of the transposed layer, so it runs on the same
+ *       kernels: the packed factors are used as they are (a row word of Ip is a column word of Ip^T).  algo:
+ *       LRBI_ALGO_AUTO, _GENERIC or _TENSOR / _TENSOR_PAIR / _TENSOR_PAIR2 (tensor-core shapes: rows % 8 == 0, and
+ *       tile_cols % 128 == 0 and tile_rows % 64 == 0 unless the grid has one tile in that direction).
+ * lrbi_masked_gemm_dw   dY [batch][rows], X [batch][cols] -> dW [rows][cols].  `workspace` is DEVICE memory of at least
+ *       lrbi_masked_gemm_dw_workspace(layout, batch) bytes, 16-byte aligned, owned by the caller, scratch for the
+ *       call (transposed copies of dY and X): the contraction runs on the tensor-core kernel with nothing pruned
+ *       inside it, and the index, decoded on the fly and never stored, is then applied to dW in place.  batch % 8 != 0
+ *       or a NULL workspace falls back to a slow one-thread-per-weight kernel.
+ * lrbi_transpose_bf16   dst [cols][rows] = transpose of src [rows][cols] (bf16 bit patterns; dst must not overlap src).
+ */
+LRBI_API lrbi_status lrbi_transpose_bf16(const uint16_t *src, int32_t rows, int32_t cols, uint16_t *dst, void *stream);
+LRBI_API lrbi_status lrbi_masked_gemm_dx(const lrbi_layout *layout, const uint16_t *Wt, const uint32_t *ip, const uint32_t *iz,
+                                         const uint16_t *dY, int32_t batch, void *dX, int32_t dx_dtype, int32_t algo, void *stream);
+LRBI_API size_t lrbi_masked_gemm_dw_workspace(const lrbi_layout *layout, int32_t batch);
+LRBI_API lrbi_status lrbi_masked_gemm_dw(const lrbi_layout *layout, const uint16_t *dY, const uint16_t *X, int32_t batch,
+                                         const uint32_t *ip, const uint32_t *iz, void *dW, int32_t dw_dtype,
+                                         void *workspace, size_t workspace_bytes, void *stream);
+
 /* Which kernel LRBI_ALGO_AUTO would run for this layout and batch (an LRBI_ALGO_* value). */
 LRBI_API int32_t lrbi_masked_gemm_choice(const lrbi_layout *layout, int32_t batch);
 

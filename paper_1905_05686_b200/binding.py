@@ -103,6 +103,14 @@ def lib():
         L.lrbi_masked_gemm_ranked.restype = i32
         L.lrbi_decode_mask_batch.argtypes = [i32, lp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         L.lrbi_decode_mask_batch.restype = i32
+        L.lrbi_transpose_bf16.argtypes = [vp, i32, i32, vp, vp]
+        L.lrbi_transpose_bf16.restype = i32
+        L.lrbi_masked_gemm_dx.argtypes = [lp, vp, vp, vp, vp, i32, vp, i32, i32, vp]
+        L.lrbi_masked_gemm_dx.restype = i32
+        L.lrbi_masked_gemm_dw_workspace.argtypes = [lp, i32]
+        L.lrbi_masked_gemm_dw_workspace.restype = ctypes.c_size_t
+        L.lrbi_masked_gemm_dw.argtypes = [lp, vp, vp, i32, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
+        L.lrbi_masked_gemm_dw.restype = i32
         L.lrbi_launch_count.argtypes = []
         L.lrbi_launch_count.restype = ctypes.c_uint64
         L.lrbi_device_status.argtypes = [i32]
@@ -239,6 +247,54 @@ def lrbi_decode_mask_batch(layers, ips, izs, stream=None):
     if rc != OK:
         raise LrbiError(rc, "lrbi_decode_mask_batch")
     return masks
+
+
+def lrbi_transpose_bf16(src: torch.Tensor, dst: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """dst [cols, rows] = src [rows, cols] transposed (bf16)."""
+    rows, cols = src.shape
+    if dst is None:
+        dst = torch.empty((cols, rows), dtype=torch.bfloat16, device=src.device)
+    rc = lib().lrbi_transpose_bf16(_dev(src, torch.bfloat16, "src"), rows, cols, _dev(dst, torch.bfloat16, "dst"), _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_transpose_bf16")
+    return dst
+
+
+def lrbi_masked_gemm_dx(layer, Wt, ip, iz, dY, dX=None, dtype=torch.bfloat16, algo=ALGO_AUTO, stream=None) -> torch.Tensor:
+    """dX = dY (W .* Ia): Wt [cols, rows] is W transposed, dY [batch, rows]; returns dX [batch, cols]."""
+    lay = Layout.of(layer)
+    if tuple(Wt.shape) != (lay.cols, lay.rows) or dY.dim() != 2 or dY.shape[1] != lay.rows:
+        raise ValueError("Wt / dY shapes do not match the layout")
+    batch = dY.shape[0]
+    if dX is None:
+        dX = torch.empty((batch, lay.cols), dtype=dtype, device=dY.device)
+    rc = lib().lrbi_masked_gemm_dx(ctypes.byref(lay), _dev(Wt, torch.bfloat16, "Wt"), _dev(ip, torch.int32, "ip"), _dev(iz, torch.int32, "iz"),
+                                   _dev(dY, torch.bfloat16, "dY"), batch, _dev(dX, dX.dtype, "dX"),
+                                   Y_F32 if dX.dtype == torch.float32 else Y_BF16, algo, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_masked_gemm_dx")
+    return dX
+
+
+def lrbi_masked_gemm_dw(layer, dY, X, ip, iz, dW=None, dtype=torch.bfloat16, workspace="auto", stream=None) -> torch.Tensor:
+    """dW = (dY^T X) .* Ia: dY [batch, rows], X [batch, cols]; returns dW [rows, cols].  workspace: a uint8 CUDA tensor of
+    at least masked_gemm_dw_workspace bytes, "auto" (one is made for the call) or None (the slow any-shape kernel)."""
+    lay = Layout.of(layer)
+    batch = dY.shape[0]
+    if tuple(dY.shape) != (batch, lay.rows) or tuple(X.shape) != (batch, lay.cols):
+        raise ValueError("dY / X shapes do not match the layout")
+    if dW is None:
+        dW = torch.empty((lay.rows, lay.cols), dtype=dtype, device=dY.device)
+    need = lib().lrbi_masked_gemm_dw_workspace(ctypes.byref(lay), batch)
+    if isinstance(workspace, str):
+        workspace = torch.empty(need, dtype=torch.uint8, device=dY.device)
+    wptr, wbytes = (ctypes.c_void_p(workspace.data_ptr()), workspace.numel()) if workspace is not None else (ctypes.c_void_p(0), 0)
+    rc = lib().lrbi_masked_gemm_dw(ctypes.byref(lay), _dev(dY, torch.bfloat16, "dY"), _dev(X, torch.bfloat16, "X"), batch,
+                                   _dev(ip, torch.int32, "ip"), _dev(iz, torch.int32, "iz"), _dev(dW, dW.dtype, "dW"),
+                                   Y_F32 if dW.dtype == torch.float32 else Y_BF16, wptr, wbytes, _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_masked_gemm_dw")
+    return dW
 
 
 def lrbi_threshold_pack(layer, mp: torch.Tensor, mz: torch.Tensor, tp: torch.Tensor, tz: torch.Tensor, stream=None):

@@ -244,6 +244,84 @@ lrbi_status lrbi_decode_mask_batch(int32_t n, const lrbi_layout *layouts, const 
     return st;
 }
 
+lrbi_status lrbi_transpose_bf16(const uint16_t *src, int32_t rows, int32_t cols, uint16_t *dst, void *stream)
+{
+    if (!src || !dst || rows < 1 || cols < 1) return LRBI_ERR_INVALID_ARG;
+    return launch_transpose_bf16(src, rows, cols, dst, static_cast<cudaStream_t>(stream));
+}
+
+// Geometry of the transposed layer: rows and columns, tile sides and grid swapped; tile (tr', tc') of it is tile
+// (tc', tr') of the layer, i.e. number tc' * GC + tr' of the factor arrays.
+static Geo transposed_geo(const Geo &g)
+{
+    Geo t = g;
+    t.rows = g.cols; t.cols = g.rows; t.tm = g.tn; t.tn = g.tm; t.gr = g.gc; t.gc = g.gr;
+    t.pitch = (t.cols + 31) / 32;
+    t.ts_r = 1; t.ts_c = g.gc;
+    return t;
+}
+
+lrbi_status lrbi_masked_gemm_dx(const lrbi_layout *layout, const uint16_t *Wt, const uint32_t *ip, const uint32_t *iz,
+                                const uint16_t *dY, int32_t batch, void *dX, int32_t dx_dtype, int32_t algo, void *stream)
+{
+    if (!layout_ok(layout) || !Wt || !ip || !iz || !dY || !dX || batch < 1) return LRBI_ERR_INVALID_ARG;
+    if (dx_dtype != LRBI_Y_BF16 && dx_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(Wt) || !aligned16(ip) || !aligned16(iz) || !aligned16(dY) || !aligned16(dX)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    const Geo t = transposed_geo(make_geo(*layout));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const TileRanks none = {nullptr, nullptr, nullptr};
+    if (algo == LRBI_ALGO_AUTO) algo = gemm_tc_supported(t, batch) ? LRBI_ALGO_TENSOR : LRBI_ALGO_GENERIC;
+    // the transposed layer's "Ip" is Iz (its rows are the layer's columns) and the other way round
+    switch (algo) {
+    case LRBI_ALGO_GENERIC: return launch_gemm_ranked_generic(t, none, Wt, iz, ip, dY, batch, dX, dx_dtype, s);
+    case LRBI_ALGO_TENSOR: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 0);
+    case LRBI_ALGO_TENSOR_PAIR: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 1);
+    case LRBI_ALGO_TENSOR_PAIR2: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 2);
+    default: return LRBI_ERR_INVALID_ARG;
+    }
+}
+
+static size_t round16(size_t b) { return (b + 15) & ~(size_t)15; }
+
+size_t lrbi_masked_gemm_dw_workspace(const lrbi_layout *layout, int32_t batch)
+{
+    if (!layout_ok(layout) || batch < 1) return 0;
+    // dY^T, X^T, and the two all-ones factors of the rank-one index the contraction runs with
+    return round16((size_t)layout->rows * batch * 2) + round16((size_t)layout->cols * batch * 2) +
+           round16((size_t)layout->cols * 4) + round16((size_t)batch * 4);
+}
+
+lrbi_status lrbi_masked_gemm_dw(const lrbi_layout *layout, const uint16_t *dY, const uint16_t *X, int32_t batch,
+                                const uint32_t *ip, const uint32_t *iz, void *dW, int32_t dw_dtype, void *workspace,
+                                size_t workspace_bytes, void *stream)
+{
+    if (!layout_ok(layout) || !dY || !X || !ip || !iz || !dW || batch < 1) return LRBI_ERR_INVALID_ARG;
+    if (dw_dtype != LRBI_Y_BF16 && dw_dtype != LRBI_Y_F32) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(ip) || !aligned16(iz) || !aligned16(dW) || !aligned16(workspace)) return LRBI_ERR_INVALID_ARG;
+    if (workspace && workspace_bytes < lrbi_masked_gemm_dw_workspace(layout, batch)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    const Geo g = make_geo(*layout);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the contraction as a forward product: "weights" X^T [cols][batch], "activations" dY^T [rows][batch], one tile of rank one
+    lrbi_layout one = {layout->cols, batch, layout->cols, batch, 1};
+    const Geo g1 = make_geo(one);
+    if (!workspace || (batch % 8) != 0 || !gemm_tc_supported(g1, layout->rows))
+        return launch_dw_generic(g, dY, X, batch, ip, iz, dW, dw_dtype, s);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    uint16_t *dYt = reinterpret_cast<uint16_t *>(ws);
+    uint16_t *Xt = reinterpret_cast<uint16_t *>(ws + round16((size_t)layout->rows * batch * 2));
+    uint32_t *ones_ip = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(Xt) + round16((size_t)layout->cols * batch * 2));
+    uint32_t *ones_iz = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(ones_ip) + round16((size_t)layout->cols * 4));
+    lrbi_status st = launch_transpose_bf16(dY, batch, layout->rows, dYt, s);
+    if (st == LRBI_OK) st = launch_transpose_bf16(X, batch, layout->cols, Xt, s);
+    if (st == LRBI_OK) st = launch_fill_words(ones_ip, (size_t)layout->cols, 1u, s);
+    if (st == LRBI_OK) st = launch_fill_words(ones_iz, (size_t)batch, 1u, s);
+    if (st == LRBI_OK) st = launch_gemm_tc(g1, Xt, ones_ip, ones_iz, dYt, layout->rows, dW, dw_dtype, s);
+    if (st == LRBI_OK) st = launch_apply_index(g, ip, iz, dW, dw_dtype, s);
+    return st;
+}
+
 uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t lrbi_device_status(int32_t clear)

@@ -162,7 +162,7 @@ __device__ __forceinline__ void panel_tile(const Geo &g, const TileRanks &rk, co
                                            int c0, int o0, int &k, int &kw, const uint32_t *&ipt, const uint32_t *&izt)
 {
     const int tr = min(o0, g.rows - 1) / g.tm, tc = min(c0, g.cols - 1) / g.tn;
-    const size_t tile = (size_t)tr * g.gc + tc;
+    const size_t tile = (size_t)tr * g.ts_r + (size_t)tc * g.ts_c;
     if (rk.ranks) {
         k = __ldg(rk.ranks + tile);
         kw = (k + 31) >> 5;
@@ -458,7 +458,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             // rank of the panel's tile (the layout's, or the tile's own in a ranked layout)
             int kp = g.k, kwp = g.kw;
             if (rk.ranks) {
-                kp = __ldg(rk.ranks + (size_t)min(tr, g.gr - 1) * g.gc + min(c0, g.cols - 1) / g.tn);
+                kp = __ldg(rk.ranks + (size_t)min(tr, g.gr - 1) * g.ts_r + (size_t)(min(c0, g.cols - 1) / g.tn) * g.ts_c);
                 kwp = (kp + 31) >> 5;
             }
             const uint32_t tail = tail_mask(kp);

@@ -16,6 +16,8 @@ struct Geo {
     int k, kw;        // rank, words per packed row/column
     int gr, gc;       // tile grid
     int pitch;        // mask words per row = ceil(cols / 32)
+    int ts_r, ts_c;   // tile (tr, tc) is tile number tr * ts_r + tc * ts_c of the factor arrays: (gc, 1), or (1, gr) when the
+                      // layer is used transposed (backward pass); only the kernels that serve that pass look at them
 };
 
 inline Geo make_geo(const lrbi_layout &l)
@@ -26,6 +28,7 @@ inline Geo make_geo(const lrbi_layout &l)
     g.gr = (l.rows + l.tile_rows - 1) / l.tile_rows;
     g.gc = (l.cols + l.tile_cols - 1) / l.tile_cols;
     g.pitch = (l.cols + 31) / 32;
+    g.ts_r = g.gc; g.ts_c = 1;
     return g;
 }
 
@@ -154,6 +157,13 @@ lrbi_status launch_decode_batch(int n, const Geo *g, const uint32_t *const *ip, 
                                 uint32_t *const *mask, cudaStream_t s);
 lrbi_status launch_gemm_ranked_generic(const Geo &g, const TileRanks &rk, const uint16_t *W, const uint32_t *ip,
                                        const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s);
+
+// Backward pass of the masked layer.
+lrbi_status launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst, cudaStream_t s);
+lrbi_status launch_apply_index(const Geo &g, const uint32_t *ip, const uint32_t *iz, void *data, int dtype, cudaStream_t s);
+lrbi_status launch_fill_words(uint32_t *dst, size_t n, uint32_t value, cudaStream_t s);
+lrbi_status launch_dw_generic(const Geo &g, const uint16_t *dY, const uint16_t *X, int batch, const uint32_t *ip,
+                              const uint32_t *iz, void *dW, int dtype, cudaStream_t s);
 
 // Inner loop of Algorithm 1.
 lrbi_status launch_threshold_pack(const Geo &g, const float *mp, const float *mz, const float *tp, const float *tz,

@@ -165,7 +165,7 @@ gemm_ranked_kernel(Geo g, TileRanks rk, const uint16_t *__restrict__ W, const ui
     for (int tc = 0; tc < g.gc; ++tc) {
         int k, kw;
         const uint32_t *ipt, *izt;
-        tile_factors(g, rk, (long long)tr * g.gc + tc, k, kw, ip, iz, ipt, izt);
+        tile_factors(g, rk, (long long)tr * g.ts_r + (long long)tc * g.ts_c, k, kw, ip, iz, ipt, izt);
         const uint32_t tail = tail_mask(k);
         const uint32_t *ipw = ipt + (long long)i * kw;
         const int c_end = min(g.tn, g.cols - tc * g.tn);
