@@ -45,7 +45,8 @@ NCU_TRAFFIC_BYTES = {
 # The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
 # batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
 OTHER_WORKLOADS = [("lenet_fc1", 32), ("decode_4096", 0), ("decode_32768", 0), ("alexnet_fc", 1), ("alexnet_fc", 16),
-                   ("alexnet_fc", 128), ("conv3x3_256", 12544), ("alexnet_fc", -1), ("ffn_16384x4096", -1)]
+                   ("alexnet_fc", 128), ("conv3x3_256", 12544), ("alexnet_fc", -1), ("ffn_16384x4096", -1),
+                   ("ffn_16384x4096", -2), ("ffn_16384x4096", -3)]   # -2: dX, -3: dW of the masked backward pass
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -227,7 +228,8 @@ def kernel_label(B, layer, batch):
     if not batch:
         return "decode"
     if batch < 0:
-        return "index_cost"
+        return {-1: "index_cost", -2: "backward dX (forward kernel on the transposed layer)",
+                -3: "backward dW (2 transposes + tensor-core product + index applied in place)"}[batch]
     plan = B.masked_gemm_plan(layer, batch)
     name = B.ALGO_NAMES[plan.algo]
     if plan.algo == B.ALGO_TENSOR:
@@ -242,7 +244,8 @@ def setup_workload(B, workload, batch, rank=0):
 
     layer = synth.CONFIGS[workload]
     decode_only = not layer.batches
-    cost_only = batch is not None and batch < 0
+    special = batch if (batch is not None and batch < 0) else 0
+    cost_only = special == -1
     batch = 0 if decode_only else (batch or layer.batches[-1])
     Ip, Iz = synth.make_factors(layer)
     ipw, izw = synth.pack_ip(Ip), synth.pack_iz(Iz)
@@ -252,6 +255,24 @@ def setup_workload(B, workload, batch, rank=0):
         out = torch.empty((layer.rows, (layer.cols + 31) // 32), dtype=torch.int32, device="cuda")
         w.update(step=lambda: B.lrbi_decode_mask(layer, ip, iz, out), out=out,
                  work_bytes=decode_bytes(layer), work_flops=0)
+    elif special in (-2, -3):
+        nb = layer.batches[-1]
+        Wb = synth.make_weights(layer)
+        Xb = synth.make_activations(layer, nb)
+        dYb = synth.make_activations(synth.Layer("dy_" + layer.name, layer.cols, layer.rows, layer.tile_cols, layer.tile_rows,
+                                                 layer.rank, layer.density), nb)
+        X, dY = B.to_device_bf16(Xb), B.to_device_bf16(dYb)
+        flops = dense_flops(layer, nb)
+        if special == -2:
+            Wt = B.lrbi_transpose_bf16(B.to_device_bf16(Wb))
+            out = torch.empty((nb, layer.cols), dtype=torch.bfloat16, device="cuda")
+            w.update(step=lambda: B.lrbi_masked_gemm_dx(layer, Wt, ip, iz, dY, dX=out), out=out, work_flops=flops,
+                     work_bytes=algorithmic_bytes(layer, nb))
+        else:
+            ws = torch.empty(B.lib().lrbi_masked_gemm_dw_workspace(__import__("ctypes").byref(B.Layout.of(layer)), nb), dtype=torch.uint8, device="cuda")
+            out = torch.empty((layer.rows, layer.cols), dtype=torch.bfloat16, device="cuda")
+            w.update(step=lambda: B.lrbi_masked_gemm_dw(layer, dY, X, ip, iz, dW=out, workspace=ws), out=out, work_flops=flops,
+                     work_bytes=2 * nb * (layer.rows + layer.cols) + 2 * layer.rows * layer.cols)
     elif cost_only:
         gr, gc = layer.grid
         W = B.to_device_bf16(synth.make_weights(layer))
