@@ -17,6 +17,7 @@ Inner loop of Algorithm 1 (Section 2.1), in lrbi_alg1_oracle.c and, for the sear
   index_cost           per tile: ones of I and of Ia, and Cost = sum of |W| where I = 1 and Ia = 0.
   sz_from_eq7          the inversion of Eq. 7 printed under it.
   threshold_for_sparsity, alg1_search   the S_p sweep with the S_z search, in the order of Algorithm 1.
+  nmf_multiplicative   the NMF of |W| that Algorithm 1 starts from, tile by tile, by multiplicative updates.
 """
 from __future__ import annotations
 
@@ -280,3 +281,33 @@ def alg1_search(W_bits: np.ndarray, theta: float, Mp: np.ndarray, Mz: np.ndarray
         if best is None or best["cost"] > cand["cost"]:  # "if Cost_min > Cost"
             best = cand
     return {"S": S, "best": best, "tried": tried}
+
+
+def nmf_multiplicative(W_bits: np.ndarray, Mp0: np.ndarray, Mz0: np.ndarray, tm: int, tn: int, iterations: int,
+                       eps: float = 1e-9):
+    """NMF of the magnitude matrix M = |W|, every tile on its own (Section 3.1), from given starting factors.
+
+    The paper hands M to "an NMF library" and names no solver; the reading taken is the multiplicative update
+    rule for the Frobenius objective ||M - Mp Mz||^2 that the paper's NMF reference gives: per iteration, first
+        Mz <- Mz * (Mp^T M) / (Mp^T Mp Mz + eps)      then, with the new Mz,      Mp <- Mp * (M Mz^T) / (Mp Mz Mz^T + eps).
+    W_bits: uint16 [rows, cols]; Mp0: [tiles, tm, k]; Mz0: [tiles, k, tn] (tiles in row-major grid order); positions of
+    an edge tile outside the matrix count as zeros of M.  Plain numpy in fp64.  Returns (Mp, Mz)."""
+    W_bits = _c(W_bits, np.uint16)
+    rows, cols = W_bits.shape
+    gr, gc = _grid(rows, cols, tm, tn)
+    M_all = np.abs(bf16_to_f64(W_bits))
+    Mp = np.array(Mp0, dtype=np.float64).copy()
+    Mz = np.array(Mz0, dtype=np.float64).copy()
+    if Mp.shape[0] != gr * gc or Mz.shape[0] != gr * gc or Mp.shape[1] != tm or Mz.shape[2] != tn or Mp.shape[2] != Mz.shape[1]:
+        raise ValueError("factor shapes do not match the tile grid")
+    for t in range(gr * gc):
+        tr, tc = divmod(t, gc)
+        M = np.zeros((tm, tn))
+        blk = M_all[tr * tm:(tr + 1) * tm, tc * tn:(tc + 1) * tn]
+        M[:blk.shape[0], :blk.shape[1]] = blk
+        P, Z = Mp[t], Mz[t]
+        for _ in range(iterations):
+            Z = Z * (P.T @ M) / (P.T @ P @ Z + eps)
+            P = P * (M @ Z.T) / (P @ (Z @ Z.T) + eps)
+        Mp[t], Mz[t] = P, Z
+    return Mp, Mz

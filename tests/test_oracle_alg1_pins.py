@@ -151,3 +151,48 @@ def test_planted_mistakes_are_caught():
     swapped = A[~I & Ia].sum()
     any_mismatch = A[I ^ Ia].sum()
     assert swapped > 0 and any_mismatch > 0                        # the oracle's 0.0 is not what these would give
+
+
+# --------------------------------------------------------------------------- NMF by multiplicative updates
+def _bits(a):
+    return synth.f32_to_bf16_bits(np.asarray(a, dtype=np.float32))
+
+
+def test_nmf_one_step_by_hand():
+    """M = [[1, 2], [2, 4]] from Mp = (1, 1)^T, Mz = (1, 1): Mz becomes (3, 6) / 2 = (1.5, 3), then Mp becomes
+    (7.5, 15) / 11.25 = (2/3, 4/3), and Mp Mz is M exactly: a rank-one matrix is recovered in one iteration."""
+    Mp, Mz = oracle.nmf_multiplicative(_bits([[1, -2], [2, 4]]), np.ones((1, 2, 1)), np.ones((1, 1, 2)), 2, 2, 1, eps=0.0)
+    assert Mz[0].tolist() == [[1.5, 3.0]]
+    assert Mp[0][:, 0] == pytest.approx([2 / 3, 4 / 3], rel=1e-15)
+    assert (Mp[0] @ Mz[0]) == pytest.approx(np.array([[1, 2], [2, 4.0]]), rel=1e-15)          # |W| is factorised, not W
+
+
+def test_nmf_properties():
+    """Non-negative factors stay non-negative, the Frobenius objective never increases (the property the update rule
+    is known for), an exact factorisation is a fixed point, and every tile is its own problem."""
+    rng = np.random.default_rng(4)
+    rows, cols, tm, tn, k = 12, 14, 6, 7, 3
+    Wb = _bits(rng.standard_normal((rows, cols)))
+    A = np.abs(synth.bf16_bits_to_f32(Wb).astype(np.float64))
+    Mp0, Mz0 = rng.random((4, tm, k)) + 0.1, rng.random((4, k, tn)) + 0.1
+    prev = None
+    for it in range(0, 6):
+        Mp, Mz = oracle.nmf_multiplicative(Wb, Mp0, Mz0, tm, tn, it)
+        assert (Mp >= 0).all() and (Mz >= 0).all()
+        err = sum(np.linalg.norm(A[tr * tm:(tr + 1) * tm, tc * tn:(tc + 1) * tn] - Mp[tr * 2 + tc] @ Mz[tr * 2 + tc]) ** 2
+                  for tr in range(2) for tc in range(2))
+        assert prev is None or err <= prev * (1 + 1e-12)
+        prev = err
+    # tile 3 alone, as a 6 x 7 matrix of its own, gives the same factors
+    Mp1, Mz1 = oracle.nmf_multiplicative(Wb[6:, 7:], Mp0[3:], Mz0[3:], tm, tn, 5)
+    assert np.allclose(Mp1[0], Mp[3], rtol=1e-13) and np.allclose(Mz1[0], Mz[3], rtol=1e-13)
+    # exact factorisation: nothing moves (values chosen exactly representable in bf16)
+    P = np.array([[1.0, 0.5], [2.0, 0.0], [0.25, 1.0]])
+    Z = np.array([[1.0, 2.0, 0.5, 0.0], [0.5, 0.0, 1.0, 2.0]])
+    Mp, Mz = oracle.nmf_multiplicative(_bits(P @ Z), P[None], Z[None], 3, 4, 3, eps=0.0)
+    assert np.allclose(Mp[0], P, rtol=1e-14) and np.allclose(Mz[0], Z, rtol=1e-14)
+    # ragged edge tiles: what lies outside the matrix counts as zero
+    Mp, Mz = oracle.nmf_multiplicative(Wb[:9, :10], Mp0, Mz0, tm, tn, 2)
+    pad = np.zeros((12, 14)); pad[:9, :10] = A[:9, :10]
+    Mp2, Mz2 = oracle.nmf_multiplicative(_bits(pad), Mp0, Mz0, tm, tn, 2)
+    assert np.allclose(Mp, Mp2) and np.allclose(Mz, Mz2)
