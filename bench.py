@@ -46,7 +46,8 @@ NCU_TRAFFIC_BYTES = {
 # batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
 OTHER_WORKLOADS = [("lenet_fc1", 32), ("decode_4096", 0), ("decode_32768", 0), ("alexnet_fc", 1), ("alexnet_fc", 16),
                    ("alexnet_fc", 128), ("conv3x3_256", 12544), ("alexnet_fc", -1), ("ffn_16384x4096", -1),
-                   ("ffn_16384x4096", -2), ("ffn_16384x4096", -3)]   # -2: dX, -3: dW of the masked backward pass
+                   ("ffn_16384x4096", -2), ("ffn_16384x4096", -3),   # -2: dX, -3: dW of the masked backward pass
+                   ("alexnet_fc", -4)]                               # -4: one iteration of the per-tile NMF of |W|
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -229,7 +230,8 @@ def kernel_label(B, layer, batch):
         return "decode"
     if batch < 0:
         return {-1: "index_cost", -2: "backward dX (forward kernel on the transposed layer)",
-                -3: "backward dW (2 transposes + tensor-core product + index applied in place)"}[batch]
+                -3: "backward dW (2 transposes + tensor-core product + index applied in place)",
+                -4: "nmf, one multiplicative update of Mz and Mp (fp32 CUDA cores)"}[batch]
     plan = B.masked_gemm_plan(layer, batch)
     name = B.ALGO_NAMES[plan.algo]
     if plan.algo == B.ALGO_TENSOR:
@@ -273,6 +275,18 @@ def setup_workload(B, workload, batch, rank=0):
             out = torch.empty((layer.rows, layer.cols), dtype=torch.bfloat16, device="cuda")
             w.update(step=lambda: B.lrbi_masked_gemm_dw(layer, dY, X, ip, iz, dW=out, workspace=ws), out=out, work_flops=flops,
                      work_bytes=2 * nb * (layer.rows + layer.cols) + 2 * layer.rows * layer.cols)
+    elif special == -4:
+        gr, gc = layer.grid
+        tiles, tm, tn, k = gr * gc, layer.tile_rows, layer.tile_cols, layer.rank
+        W = B.to_device_bf16(synth.make_weights(layer))
+        rng = np.random.default_rng(0)
+        mp = torch.from_numpy((rng.random((tiles, tm, k)) * 0.1 + 0.01).astype(np.float32)).cuda()
+        mz = torch.from_numpy((rng.random((tiles, k, tn)) * 0.1 + 0.01).astype(np.float32)).cuda()
+        ws = torch.empty(B.lib().lrbi_nmf_workspace(__import__("ctypes").byref(B.Layout.of(layer))), dtype=torch.uint8, device="cuda")
+        # two products of 2 k tm tn flops, two Gram matrices and two k-term denominators per element, per tile
+        flops = tiles * (4 * k * tm * tn + 2 * k * k * (tm + tn) + 2 * k * k * (tm + tn))
+        w.update(step=lambda: B.lrbi_nmf_update(layer, W, mp, mz, 1, workspace=ws), out=mp, work_flops=flops, alu=True,
+                 work_bytes=2 * 2 * layer.rows * layer.cols + 4 * 4 * tiles * k * (tm + tn))
     elif cost_only:
         gr, gc = layer.grid
         W = B.to_device_bf16(synth.make_weights(layer))
@@ -457,10 +471,15 @@ def run_ours(args):
             ts = time_calls(ow["step"], args.other_steps, 3, flush2)
             nl = (B.launch_count() - l0) / (args.other_steps + 3)
             ms = float(np.mean(ts))
+            rl = roofline_of(name, ow["batch"], ow["work_bytes"], ow["work_flops"], ms, peaks)
+            if ow.get("alu"):
+                # fp32 FMA roof: 148 SMs x 128 lanes x 2 flop at the maximum SM clock (1965 MHz) = 74.4 TFLOP/s
+                ach = ow["work_flops"] / (ms * 1e-3) / 1e12
+                rl = {"bound": "alu", "achieved": ach, "peak": 74.4, "unit": "TFLOP/s", "frac": ach / 74.4, "traffic": None,
+                      "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz", "kernel_ms": ms}
             others.append({"workload": name, "batch": ow["batch"], "kernel": kernel_label(B, ow["layer"], ow["batch"]),
                            "ms": ms, "ms_median": float(np.median(ts)), "launches_per_step": nl,
-                           "algorithmic_bytes": ow["work_bytes"], "dense_flops": ow["work_flops"],
-                           "roofline": roofline_of(name, ow["batch"], ow["work_bytes"], ow["work_flops"], ms, peaks)})
+                           "algorithmic_bytes": ow["work_bytes"], "dense_flops": ow["work_flops"], "roofline": rl})
             del ow
         if B.device_status() != 0:
             raise SystemExit("device status word is not clean after the other workloads: %d" % B.device_status())

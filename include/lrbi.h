@@ -262,6 +262,23 @@ LRBI_API lrbi_status lrbi_decode_mask_batch(int32_t n, const lrbi_layout *layout
                                             const uint32_t *const *iz, uint32_t *const *mask_out, void *stream);
 
 /*
+ * NMF of the magnitude matrix (Section 2.1: M[i][j] = |W[i][j]| "is factorized by an NMF library" into Mp, Mz,
+ * Eq. 4; first two steps of Algorithm 1), every tile on its own (Section 3.1).  The paper names no solver; this is
+ * the multiplicative update rule for the Frobenius objective ||M - Mp Mz||^2 of the NMF reference it cites, from
+ * the caller's starting factors: per iteration
+ *       Mz <- Mz * (Mp^T M) / (Mp^T Mp Mz + eps),   then   Mp <- Mp * (M Mz^T) / (Mp Mz Mz^T + eps),
+ * in fp32.  Positions of an edge tile outside the matrix count as zeros of M.  rank <= 256.
+ *   W     device, bf16 bit patterns, [rows][cols]
+ *   mp    device, fp32, [GR*GC][tile_rows][rank], in and out (start from positive values)
+ *   mz    device, fp32, [GR*GC][rank][tile_cols], in and out
+ *   workspace   device, lrbi_nmf_workspace(layout) bytes, 16-byte aligned, scratch for the call
+ * The results feed lrbi_threshold_pack.
+ */
+LRBI_API size_t lrbi_nmf_workspace(const lrbi_layout *layout);
+LRBI_API lrbi_status lrbi_nmf_update(const lrbi_layout *layout, const uint16_t *W, float *mp, float *mz, int32_t iterations,
+                                     float eps, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Backward pass of the masked layer (Section 2.2: the pruned network is retrained "using a masking layer" Ia, so
  * gradients flow through kept weights only).  With Y = X (W .* Ia)^T and dY = dL/dY [batch][rows]:
  *       dX[b][i] = sum_o  Ia[o][i] ? dY[b][o] * W[o][i] : 0          dW[o][i] = Ia[o][i] ? sum_b dY[b][o] * X[b][i] : 0

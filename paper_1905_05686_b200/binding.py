@@ -111,6 +111,10 @@ def lib():
         L.lrbi_masked_gemm_dw_workspace.restype = ctypes.c_size_t
         L.lrbi_masked_gemm_dw.argtypes = [lp, vp, vp, i32, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
         L.lrbi_masked_gemm_dw.restype = i32
+        L.lrbi_nmf_workspace.argtypes = [lp]
+        L.lrbi_nmf_workspace.restype = ctypes.c_size_t
+        L.lrbi_nmf_update.argtypes = [lp, vp, vp, vp, i32, ctypes.c_float, vp, ctypes.c_size_t, vp]
+        L.lrbi_nmf_update.restype = i32
         L.lrbi_launch_count.argtypes = []
         L.lrbi_launch_count.restype = ctypes.c_uint64
         L.lrbi_device_status.argtypes = [i32]
@@ -295,6 +299,19 @@ def lrbi_masked_gemm_dw(layer, dY, X, ip, iz, dW=None, dtype=torch.bfloat16, wor
     if rc != OK:
         raise LrbiError(rc, "lrbi_masked_gemm_dw")
     return dW
+
+
+def lrbi_nmf_update(layer, W, mp, mz, iterations, eps=1e-9, workspace=None, stream=None):
+    """In-place multiplicative NMF updates of (mp, mz) towards |W|, tile by tile; returns (mp, mz)."""
+    lay = Layout.of(layer)
+    need = lib().lrbi_nmf_workspace(ctypes.byref(lay))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=W.device)
+    rc = lib().lrbi_nmf_update(ctypes.byref(lay), _dev(W, torch.bfloat16, "W"), _dev(mp, torch.float32, "mp"), _dev(mz, torch.float32, "mz"),
+                               iterations, ctypes.c_float(eps), ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream_ptr(stream))
+    if rc != OK:
+        raise LrbiError(rc, "lrbi_nmf_update")
+    return mp, mz
 
 
 def lrbi_threshold_pack(layer, mp: torch.Tensor, mz: torch.Tensor, tp: torch.Tensor, tz: torch.Tensor, stream=None):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblrbi.so")
-SOURCES = ["api.cu", "decode_kernels.cu", "gemv_kernels.cu", "gemm_tc.cu", "alg1_kernels.cu", "ranked_kernels.cu", "backward_kernels.cu"]
+SOURCES = ["api.cu", "decode_kernels.cu", "gemv_kernels.cu", "gemm_tc.cu", "alg1_kernels.cu", "ranked_kernels.cu", "backward_kernels.cu", "nmf_kernels.cu"]
 
 
 def _stale() -> bool:

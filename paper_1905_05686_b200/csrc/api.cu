@@ -322,6 +322,20 @@ lrbi_status lrbi_masked_gemm_dw(const lrbi_layout *layout, const uint16_t *dY, c
     return st;
 }
 
+size_t lrbi_nmf_workspace(const lrbi_layout *layout)
+{
+    return layout_ok(layout) ? nmf_workspace_bytes(make_geo(*layout)) : 0;
+}
+
+lrbi_status lrbi_nmf_update(const lrbi_layout *layout, const uint16_t *W, float *mp, float *mz, int32_t iterations, float eps,
+                            void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!layout_ok(layout) || !W || !mp || !mz || !workspace || iterations < 0 || !(eps >= 0.f)) return LRBI_ERR_INVALID_ARG;
+    if (!aligned16(workspace) || workspace_bytes < lrbi_nmf_workspace(layout)) return LRBI_ERR_INVALID_ARG;
+    if (device_timeout_seen()) return LRBI_ERR_TIMEOUT;
+    return launch_nmf(make_geo(*layout), W, mp, mz, iterations, eps, static_cast<float *>(workspace), static_cast<cudaStream_t>(stream));
+}
+
 uint64_t lrbi_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t lrbi_device_status(int32_t clear)

@@ -165,6 +165,10 @@ lrbi_status launch_fill_words(uint32_t *dst, size_t n, uint32_t value, cudaStrea
 lrbi_status launch_dw_generic(const Geo &g, const uint16_t *dY, const uint16_t *X, int batch, const uint32_t *ip,
                               const uint32_t *iz, void *dW, int dtype, cudaStream_t s);
 
+// NMF of |W| per tile (multiplicative updates).
+size_t nmf_workspace_bytes(const Geo &g);
+lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, int iterations, float eps, float *ws, cudaStream_t s);
+
 // Inner loop of Algorithm 1.
 lrbi_status launch_threshold_pack(const Geo &g, const float *mp, const float *mz, const float *tp, const float *tz,
                                   uint32_t *ip, uint32_t *iz, cudaStream_t s);
