@@ -74,6 +74,10 @@ nmf_gemm_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__
 }
 
 // G[a][b] = sum_r F(r, a) F(r, b): ZMODE 0: F = Mp [tm][k] (r = row), ZMODE 1: F = Mz [k][tn] (r = column).
+// grid = (k*k / 256, layer tiles, slices of the reduction): a block sums its slice of r and adds it to G (zeroed
+// before the launch) with one atomic per entry; a lone thread per entry over the whole reduction was measured at
+// 200-280 us per launch on the AlexNet layer, as much as the large products.
+constexpr int NMF_GRAM_SLICE = 32;
 template <int ZMODE>
 __global__ void __launch_bounds__(256)
 nmf_gram_kernel(Geo g, const float *__restrict__ F, float *__restrict__ G)
@@ -84,10 +88,11 @@ nmf_gram_kernel(Geo g, const float *__restrict__ F, float *__restrict__ G)
     const int a = e / k, b = e - a * k;
     const float *Ft = F + (size_t)tile * (ZMODE == 0 ? (size_t)g.tm * k : (size_t)k * g.tn);
     const int R = ZMODE == 0 ? g.tm : g.tn;
+    const int r0 = blockIdx.z * NMF_GRAM_SLICE, r1 = min(R, r0 + NMF_GRAM_SLICE);
     float s = 0.f;
-    for (int r = 0; r < R; ++r)
+    for (int r = r0; r < r1; ++r)
         s = ZMODE == 0 ? fmaf(Ft[(size_t)r * k + a], Ft[(size_t)r * k + b], s) : fmaf(Ft[(size_t)a * g.tn + r], Ft[(size_t)b * g.tn + r], s);
-    G[(size_t)tile * k * k + e] = s;
+    atomicAdd(G + (size_t)tile * k * k + e, s);
 }
 
 constexpr int NMF_MAX_RANK = 256;
@@ -141,10 +146,12 @@ lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, in
     const unsigned kt = (unsigned)((g.k + NG_T - 1) / NG_T), gk2 = (unsigned)((g.k * g.k + 255) / 256);
     for (int it = 0; it < iterations; ++it) {
         nmf_gemm_kernel<0><<<dim3((unsigned)((g.tn + NG_T - 1) / NG_T), kt, (unsigned)tiles), 256, 0, s>>>(g, W, mp, N);
-        nmf_gram_kernel<0><<<dim3(gk2, (unsigned)tiles), 256, 0, s>>>(g, mp, G);
+        cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
+        nmf_gram_kernel<0><<<dim3(gk2, (unsigned)tiles, (unsigned)((g.tm + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mp, G);
         nmf_update_z_kernel<<<dim3((unsigned)((g.tn + 127) / 128), (unsigned)tiles), 128, 0, s>>>(g, N, G, mz, eps);
         nmf_gemm_kernel<1><<<dim3(kt, (unsigned)((g.tm + NG_T - 1) / NG_T), (unsigned)tiles), 256, 0, s>>>(g, W, mz, N);
-        nmf_gram_kernel<1><<<dim3(gk2, (unsigned)tiles), 256, 0, s>>>(g, mz, G);
+        cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
+        nmf_gram_kernel<1><<<dim3(gk2, (unsigned)tiles, (unsigned)((g.tn + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mz, G);
         nmf_update_p_kernel<<<dim3((unsigned)((g.tm + 127) / 128), (unsigned)tiles), 128, 0, s>>>(g, N, G, mp, eps);
         count_launch(6);
     }
