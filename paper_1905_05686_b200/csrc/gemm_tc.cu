@@ -220,6 +220,7 @@ struct TcCtl {
     uint64_t masked[8];      // ... and its W tile has been pruned in place (leader of a pair: in both CTAs)
     uint64_t empty[8];       // the MMAs that read the stage have completed
     uint64_t accum;
+    uint64_t tmem_free;      // PERSIST: tensor memory may be overwritten by the next tile's MMAs
     uint64_t epi;            // the eight pruning warps meet here before the epilogue's copy-out
     uint64_t bits_ready[2];  // decoders -> pruners: the index bits of a panel are in buffer b
     uint64_t bits_free[2];   // pruners -> decoders: buffer b may be overwritten
@@ -271,7 +272,12 @@ __device__ __forceinline__ int warp_of_thread_decoder_group(unsigned tid)
 // once per 256 rows of W instead of once per 128, and each byte of it is read from shared memory by
 // one tensor core pass instead of two.  Two such blocks are resident per SM (three stages each), so
 // one block's epilogue and panel hand-overs overlap the other's MMAs.
-template <int BN, int PW, bool PAIR>
+// PERSIST (two-accumulator pairs, K not split): the grid is one pair per two SMs and a pair walks output tiles
+// (pair p takes tiles p, p + pairs, ...).  Stage, panel and barrier state run on across tiles, so while the pruning
+// warps drain tensor memory of tile n (through warp-private staging, the operand stages are no longer free), the
+// copies, the factor words and the first index panels of tile n + 1 are already on their way; the first MMA of a
+// tile waits until both CTAs have emptied tensor memory.
+template <int BN, int PW, bool PAIR, bool PERSIST>
 __global__ void __launch_bounds__(tc_threads(BN), BN > 256 ? 1 : 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g, TileRanks rk,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
@@ -302,7 +308,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     uint32_t *planes = row_bits + 2 * TC_BM * PW + dgrp * dgroup_words;
     uint32_t *iz_stage = planes + g.kw * 32 * PWS;
     uint32_t *ip_stage = iz_stage + PW * 32 * g.kw;
-    TcCtl *ctl = reinterpret_cast<TcCtl *>(row_bits + 2 * TC_BM * PW + NDG * dgroup_words);
+    uint8_t *epi_stage = reinterpret_cast<uint8_t *>(row_bits + 2 * TC_BM * PW + NDG * dgroup_words);   // PERSIST: 1 KB per pruning warp
+    TcCtl *ctl = reinterpret_cast<TcCtl *>(epi_stage + (PERSIST ? TC_MASK_WARPS * 1024 : 0));
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -313,8 +320,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u; // 0 = leader of the pair
     // grid.x runs fastest over blocks that share rows of W, so W streams from HBM once and X stays in L2.
     // Pair mode: the two CTAs of a cluster are neighbours along x (x = 2 * batch tile + rank), y = 256-row pair.
-    const int b0 = (PAIR ? (blockIdx.x >> 1) : blockIdx.x) * BN;                       // first batch row of the tile
-    const int o0 = (PAIR ? (blockIdx.y * 2 + (int)rank) : blockIdx.y) * TC_BM;          // first row of W of this block
+    // PERSIST: the block's n-th tile is tile t = (pair index) + n * (pairs in the grid); t runs fastest over batch tiles.
+    const int nbt = (batch + BN - 1) / BN;
+    const int tile_first = PERSIST ? (int)(blockIdx.x >> 1) : 0, tile_step = PERSIST ? (int)(gridDim.x >> 1) : 1;
+    const int my_tiles = PERSIST ? (nbt * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) - tile_first + tile_step - 1) / tile_step : 1;
+    auto tile_b0 = [&](int n) {                          // first batch row of the block's n-th tile
+        return PERSIST ? ((tile_first + n * tile_step) % nbt) * BN : (int)(PAIR ? (blockIdx.x >> 1) : blockIdx.x) * BN;
+    };
+    auto tile_o0 = [&](int n) {                          // first row of W of this block in its n-th tile
+        return PERSIST ? (((tile_first + n * tile_step) / nbt) * 2 + (int)rank) * TC_BM
+                       : (int)(PAIR ? (blockIdx.y * 2 + rank) : blockIdx.y) * TC_BM;
+    };
+    const int b0 = tile_b0(0), o0 = tile_o0(0);
     const int nkb_total = (g.cols + TC_BK - 1) / TC_BK;
     const int kb_begin = blockIdx.z * kb_per_split;      // a multiple of KBP
     const int kb_end = min(nkb_total, kb_begin + kb_per_split);
@@ -322,9 +339,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
 
     // Long-latency requests first: the decoder warps ask for the factor words of their first panel, one
     // thread warms the TMA descriptors; both overlap the barrier and tensor-memory set-up below.
-    if (warp >= 2 + TC_MASK_WARPS && dgrp * KBP < nkb)   // group g starts with panel g
-        stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + dgrp * KBP) * TC_BK, o0,
-                            (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1), TC_DECODE_WARPS * 32);
+    {
+        const int npanels0 = (nkb + KBP - 1) / KBP;      // group g starts with panel g (of the block's first tiles)
+        if (warp >= 2 + TC_MASK_WARPS && dgrp < my_tiles * npanels0)
+            stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + (dgrp % npanels0) * KBP) * TC_BK,
+                                tile_o0(dgrp / npanels0),
+                                (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1), TC_DECODE_WARPS * 32);
+    }
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&w_map) : "memory");
@@ -338,6 +359,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         }
         mbar_init(&ctl->accum, 1);
         mbar_init(&ctl->epi, TC_MASK_WARPS);
+        mbar_init(&ctl->tmem_free, 2 * TC_MASK_WARPS);   // PERSIST, leader: the pruning warps of both CTAs have drained tensor memory
         for (int b = 0; b < 2; ++b) {
             mbar_init(&ctl->bits_ready[b], TC_DECODE_WARPS);
             mbar_init(&ctl->bits_free[b], TC_MASK_WARPS);
@@ -362,8 +384,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             bool issued = false;
             int s = 0;
             uint32_t parity = 1;                        // a fresh barrier reports its "previous" phase complete
+            bool go = true;
+            for (int n = 0; n < my_tiles && go; ++n) {
+            const int b0 = tile_b0(n), o0 = tile_o0(n);
             for (int it = 0; it < nkb; ++it) {
-                if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) break;
+                if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) { go = false; break; }
                 mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES + TC_A_STAGE_BYTES);
                 tma_load_2d(a_base + s * TC_A_STAGE_BYTES, &w_map, &ctl->full[s], (kb_begin + it) * TC_BK, o0);
 #pragma unroll
@@ -372,6 +397,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                                 (kb_begin + it) * TC_BK, b0 + a * 256 + (int)rank * XBOX_ROWS);
                 issued = true;
                 if (++s == stages) { s = 0; parity ^= 1; }
+            }
             }
             if (*abort_flag && issued) {
                 // Abort path: copies already issued must land before this block's shared memory is
@@ -388,6 +414,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             bool ok = true;
             int s = 0;
             uint32_t parity = 0;
+            uint32_t tfree_parity = 1;                  // a fresh barrier reports its "previous" phase complete
+            for (int n = 0; n < my_tiles && ok; ++n) {
+            if (PERSIST) {                              // both CTAs have read the previous tile's accumulators
+                ok = mbar_wait(&ctl->tmem_free, tfree_parity, abort_flag, status, DEV_TIMEOUT_ACCUM);
+                tfree_parity ^= 1;
+                if (!ok) break;
+                tc_fence_after();
+            }
             for (int it = 0; it < nkb && ok; ++it) {
                 ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
@@ -413,13 +447,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             if (ok) {                                   // accumulator complete
                 if (PAIR) umma2_commit_both(&ctl->accum); else umma_commit(&ctl->accum);
             }
+            }
         } else if (lane == 0) {
             // ------------------------------------------------------------- relay (second CTA of a pair)
             // tells the leader when this CTA's half of a stage is loaded and pruned
             bool ok = true;
             int s = 0;
             uint32_t parity = 0;
-            for (int it = 0; it < nkb && ok; ++it) {
+            for (long long it = 0; it < (long long)my_tiles * nkb && ok; ++it) {
                 ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
                 mbar_arrive_remote(&ctl->masked[s], 0);
@@ -430,15 +465,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         // ------------------------------------------------------------- index decoders
         const int dt = (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1);   // 0..127: row of the block this thread decodes
         const int dw = dt >> 5;                         // decoder warp 0..3
-        const int tr = o0 / g.tm;                       // the 128 rows lie in one tile row
-        const int i0 = o0 - tr * g.tm;                  // first row of the block inside its tile
-        const bool row_ok = o0 + dt < g.rows && i0 + dt < g.tm;
         const int bit_col = column_of_bit(lane);        // column (0..31) this lane stands for in a transpose
         const int npanels = (nkb + KBP - 1) / KBP;
 
-        auto stage_factors = [&](int P) {
-            if (P < npanels)
-                stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + P * KBP) * TC_BK, o0, dt, TC_DECODE_WARPS * 32);
+        // panels are counted across the block's tiles: panel PG is panel PG % npanels of tile PG / npanels
+        auto stage_factors = [&](int PG) {
+            if (PG < my_tiles * npanels) {
+                const int n2 = PG / npanels, P2 = PG - n2 * npanels;
+                stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + P2 * KBP) * TC_BK, tile_o0(n2), dt, TC_DECODE_WARPS * 32);
+            }
         };
 
         uint32_t dsync_parity = 0;
@@ -451,8 +486,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         };
 
         // (the group's first panel was requested at kernel entry)
-        for (int P = dgrp; P < npanels && ok; P += NDG) {
-            const int buf = P & 1;
+        for (int PG = dgrp; PG < my_tiles * npanels && ok; PG += NDG) {
+            const int tile_n = PG / npanels, P = PG - tile_n * npanels;
+            const int o0 = tile_o0(tile_n);
+            const int tr = o0 / g.tm;                   // the 128 rows lie in one tile row
+            const int i0 = o0 - tr * g.tm;              // first row of the block inside its tile
+            const bool row_ok = o0 + dt < g.rows && i0 + dt < g.tm;
+            const int buf = PG & 1;
             uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
             const int c0 = (kb_begin + P * KBP) * TC_BK;
             // rank of the panel's tile (the layout's, or the tile's own in a ranked layout)
@@ -493,9 +533,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             }
             dsync();                                     // planes complete, factor staging consumed
             if (!ok) break;
-            stage_factors(P + NDG);                      // the group's next panel: its factor words start their trip now
+            stage_factors(PG + NDG);                     // the group's next panel: its factor words start their trip now
             // the pruning warps must be done with the panel that used this buffer two panels ago
-            ok = mbar_wait(&ctl->bits_free[buf], ((P >> 1) & 1) ^ 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
+            ok = mbar_wait(&ctl->bits_free[buf], ((PG >> 1) & 1) ^ 1, abort_flag, status, DEV_TIMEOUT_EMPTY);
             if (!ok) break;
             // (b) Eq. 3 for one row: OR of the planes its Ip bits select
             uint32_t acc[PW];
@@ -546,7 +586,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         int s = 0;                                       // stage of the current K block
         uint32_t full_parity = 0;
         int kp = 0;                                      // K block inside its panel
-        int P = 0;                                       // panel index inside this block's K range
+        int P = 0;                                       // panel index, counted across the block's tiles
+        for (int tile_n = 0; tile_n < my_tiles && ok; ++tile_n) {
+        const int b0 = tile_b0(tile_n), o0 = tile_o0(tile_n);
         for (int it = 0; it < nkb && ok; ++it) {
             const int buf = P & 1;
             if (kp == 0) {                               // first K block of a panel: its index bits must be there
@@ -581,10 +623,71 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             if (++s == stages) { s = 0; full_parity ^= 1; }
             if (++kp == KBP) { kp = 0; ++P; }
         }
+        if (kp != 0) { kp = 0; ++P; }                    // a tile's last panel may be short
 
         // ------------------------------------------------------------- epilogue (same warps)
-        if (ok) ok = mbar_wait(&ctl->accum, 0, abort_flag, status, DEV_TIMEOUT_ACCUM);
-        if (ok) {
+        if (ok) ok = mbar_wait(&ctl->accum, (uint32_t)(tile_n & 1), abort_flag, status, DEV_TIMEOUT_ACCUM);
+        if (ok && PERSIST) {
+            // The operand stages already belong to the next tile: every warp moves its 32 output features x 16
+            // (fp32: 8) batch columns through 1 KB of its own and stores 16-byte pieces, 64 (128) bytes of a row of Y
+            // per four (eight) lanes.
+            tc_fence_after();
+            const bool out32 = y_dtype == LRBI_Y_F32;
+            const int quad = warp & 3, half = mw >> 2;   // tensor-memory lanes this warp may read; its half of the columns
+            uint8_t *st = epi_stage + mw * 1024;
+            const int f0 = o0 + quad * 32;               // first output feature of the warp
+            const bool vec_ok = (g.rows % (out32 ? 4 : 8)) == 0;
+            for (int ch = 0; ch < BN / 32; ++ch) {
+                const int cl = half * (BN / 2) + ch * 16;            // first batch column of the chunk inside the tile
+                uint32_t v[16];
+                tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)cl, v);
+                tmem_ld_wait();
+                if (!out32) {
+                    uint16_t *s16 = reinterpret_cast<uint16_t *>(st);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) s16[j * 32 + lane] = f32_to_bf16_rne(__uint_as_float(v[j]));
+                    __syncwarp();
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int idx = lane + 32 * u, col = idx >> 2, part = idx & 3;
+                        const int bb = b0 + cl + col, ff = f0 + part * 8;
+                        if (bb < batch && ff < g.rows) {
+                            uint16_t *dst = reinterpret_cast<uint16_t *>(Y) + (size_t)bb * g.rows + ff;
+                            if (vec_ok && ff + 8 <= g.rows) *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(st + col * 64 + part * 16);
+                            else for (int e = 0; e < min(8, g.rows - ff); ++e) dst[e] = s16[col * 32 + part * 8 + e];
+                        }
+                    }
+                    __syncwarp();
+                } else {
+                    float *s32 = reinterpret_cast<float *>(st);
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) s32[j * 32 + lane] = __uint_as_float(v[hh * 8 + j]);
+                        __syncwarp();
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int idx = lane + 32 * u, col = idx >> 3, part = idx & 7;
+                            const int bb = b0 + cl + hh * 8 + col, ff = f0 + part * 4;
+                            if (bb < batch && ff < g.rows) {
+                                float *dst = reinterpret_cast<float *>(Y) + (size_t)bb * g.rows + ff;
+                                if (vec_ok && ff + 4 <= g.rows) *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(st + col * 128 + part * 16);
+                                else for (int e = 0; e < min(4, g.rows - ff); ++e) dst[e] = s32[col * 32 + part * 4 + e];
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+            // this warp has read its part of tensor memory: tell the leader's MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(&ctl->tmem_free);
+                else mbar_arrive_remote(&ctl->tmem_free, 0);
+            }
+        }
+        if (ok && !PERSIST) {
             tc_fence_after();
             // All MMAs have completed, so the operand stages are free: reuse them to transpose the
             // accumulator (lane = output feature) into rows of Y (contiguous output features).  The
@@ -652,6 +755,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 if (pass0 + PASS < BN) meet();           // staging may be overwritten by the next pass
             }
         }
+        }                                                // the block's tiles
     }
 
     tc_fence_before();
@@ -750,6 +854,8 @@ struct TcPlan {
     int stages;          // operand stages in shared memory
     size_t smem;         // dynamic shared memory per block
     size_t scratch;      // bytes of fp32 partial sums (0 when K is not split)
+    bool persist;        // one pair per two SMs walks the output tiles (two-accumulator pairs, K not split)
+    int pairs;           // persist: pairs in the grid
 };
 
 // `force`: 0 = choose by shape; 1 = CTA pairs with one accumulator (256 batch columns per pair);
@@ -808,7 +914,15 @@ static bool make_tc_plan(const Geo &g, int batch, int sm_count, int force, TcPla
     // (an SM has 228 KB of shared memory; each resident block also reserves 1 KB)
     const size_t b_stage = (size_t)(p.pair ? p.bn / 2 : p.bn) * TC_BK * 2;
     const size_t dgroup_words = (size_t)g.kw * 32 * (p.pw == 8 ? 12 : p.pw) + (size_t)p.pw * 32 * g.kw + (size_t)TC_BM * g.kw;
-    const size_t extras = ((size_t)2 * TC_BM * p.pw + tc_decode_groups(p.bn) * dgroup_words) * 4 + sizeof(TcCtl);
+    p.persist = p.pair && p.bn == 512 && p.splits == 1;
+    p.pairs = 0;
+    if (p.persist) {
+        const long long tiles2 = (long long)((batch + 511) / 512) * (p.row_blocks / 2);
+        p.pairs = (int)(tiles2 < sm_count / 2 ? tiles2 : sm_count / 2);
+        if (p.pairs < 1) p.persist = false;
+    }
+    const size_t extras = ((size_t)2 * TC_BM * p.pw + tc_decode_groups(p.bn) * dgroup_words) * 4 + sizeof(TcCtl) +
+                          (p.persist ? TC_MASK_WARPS * 1024 : 0);
     const size_t per_stage = TC_A_STAGE_BYTES + b_stage;
     const size_t half_sm = 113 * 1024, whole_sm = 224 * 1024;
     int stages = (int)((half_sm - extras) / per_stage);
@@ -832,7 +946,7 @@ static int device_sm_count(int *dev_out)
     return sm_count;
 }
 
-template <int BN, int PW, bool PAIR>
+template <int BN, int PW, bool PAIR, bool PERSIST>
 static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const uint16_t *W, const uint32_t *ip,
                              const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype,
                              cudaStream_t s, float *partials, const TileRanks &rk)
@@ -856,7 +970,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
-    auto kern = gemm_tc_kernel<BN, PW, PAIR>;
+    auto kern = gemm_tc_kernel<BN, PW, PAIR, PERSIST>;
     {
         // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the function
         static bool attr_done[LRBI_MAX_DEVICES] = {false};
@@ -869,6 +983,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     }
     const unsigned nbt = (unsigned)((batch + BN - 1) / BN);
     dim3 grid(PAIR ? 2 * nbt : nbt, (unsigned)(PAIR ? plan.row_blocks / 2 : plan.row_blocks), (unsigned)plan.splits);
+    if (PERSIST) grid = dim3(2u * (unsigned)plan.pairs, 1, 1);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(tc_threads(BN));
@@ -916,14 +1031,16 @@ static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, c
         if (!partials) { note_cuda_error((int)cudaErrorMemoryAllocation); return LRBI_ERR_CUDA; }
     }
 #define LRBI_TC_CASE(BN_, PW_, PAIR_) \
-    if (plan.bn == BN_ && plan.pw == PW_ && plan.pair == PAIR_) \
-        return launch_tc<BN_, PW_, PAIR_>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials, rk);
+    if (plan.bn == BN_ && plan.pw == PW_ && plan.pair == PAIR_ && !plan.persist) \
+        return launch_tc<BN_, PW_, PAIR_, false>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials, rk);
     LRBI_TC_CASE(16, 8, false) LRBI_TC_CASE(16, 2, false)
     LRBI_TC_CASE(32, 8, false) LRBI_TC_CASE(32, 2, false)
     LRBI_TC_CASE(64, 8, false) LRBI_TC_CASE(64, 2, false)
     LRBI_TC_CASE(128, 8, false) LRBI_TC_CASE(128, 2, false)
     LRBI_TC_CASE(256, 8, true) LRBI_TC_CASE(256, 2, true)
     LRBI_TC_CASE(512, 8, true) LRBI_TC_CASE(512, 2, true)
+    if (plan.persist && plan.pw == 8) return launch_tc<512, 8, true, true>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials, rk);
+    if (plan.persist && plan.pw == 2) return launch_tc<512, 2, true, true>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials, rk);
 #undef LRBI_TC_CASE
     return LRBI_ERR_UNSUPPORTED;
 }
