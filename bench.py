@@ -31,7 +31,7 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu capture
 # summarised under profiles/ (null for workloads without a capture of the current kernel)
 NCU_TRAFFIC_BYTES = {
-    ("ffn_16384x4096", 4096): 406_000_000,      # 290 MB read + 116 MB written (profiles/ncu_traffic_all_workloads.md)
+    ("ffn_16384x4096", 4096): 401_400_000,      # 285.8 MB read + 115.6 MB written (profiles/gemm_tc_pair2_ffn_16384x4096.md)
     ("lenet_fc1", 32): 1_050_000,
     ("decode_4096", 0): 534_000,                # the 2 MiB mask is still in L2 when the kernel ends
     ("decode_32768", 0): 104_200_000,
