@@ -315,7 +315,13 @@ lrbi_status lrbi_masked_gemm_dw(const lrbi_layout *layout, const uint16_t *dY, c
     uint32_t *ones_iz = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(ones_ip) + round16((size_t)layout->cols * 4));
     lrbi_status st = launch_transpose_bf16(dY, batch, layout->rows, dYt, s);
     if (st == LRBI_OK) st = launch_transpose_bf16(X, batch, layout->cols, Xt, s);
-    if (st == LRBI_OK) st = launch_fill_words(ones_ip, (size_t)layout->cols, 1u, s);
+    if (st != LRBI_OK) return st;
+    // First choice: the persistent pair kernel with nothing pruned inside the contraction and the index (seen transposed:
+    // rows = layer columns) applied as the output tile is stored.
+    st = launch_gemm_tc_dw(g1, transposed_geo(g), Xt, iz, ip, dYt, layout->rows, dW, dw_dtype, s);
+    if (st != LRBI_ERR_UNSUPPORTED) return st;
+    // Otherwise: the forward kernel with an all-ones index of rank one, then the index applied to dW in place.
+    st = launch_fill_words(ones_ip, (size_t)layout->cols, 1u, s);
     if (st == LRBI_OK) st = launch_fill_words(ones_iz, (size_t)batch, 1u, s);
     if (st == LRBI_OK) st = launch_gemm_tc(g1, Xt, ones_ip, ones_iz, dYt, layout->rows, dW, dw_dtype, s);
     if (st == LRBI_OK) st = launch_apply_index(g, ip, iz, dW, dw_dtype, s);

@@ -277,9 +277,13 @@ __device__ __forceinline__ int warp_of_thread_decoder_group(unsigned tid)
 // warps drain tensor memory of tile n (through warp-private staging, the operand stages are no longer free), the
 // copies, the factor words and the first index panels of tile n + 1 are already on their way; the first MMA of a
 // tile waits until both CTAs have emptied tensor memory.
-template <int BN, int PW, bool PAIR, bool PERSIST>
+// DW (persistent pairs only): the product of the masked layer's weight gradient, dW = (dY^T X) .* Ia.  Nothing is
+// pruned inside the contraction (the pruning warps only pass the stages on); `gi` is the layout of the index as the
+// output sees it (rows = rows of the output tile, columns = its batch axis), the decoders decode the two 256-column
+// panels of each output tile from it, and the epilogue zeroes the pruned outputs as it stores them.
+template <int BN, int PW, bool PAIR, bool PERSIST, bool DW>
 __global__ void __launch_bounds__(tc_threads(BN), BN > 256 ? 1 : 2)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g, TileRanks rk,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g, Geo gi, TileRanks rk,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
                int stages, int *status)
@@ -303,11 +307,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     uint32_t *row_bits = reinterpret_cast<uint32_t *>(b_base + (size_t)stages * B_STAGE_BYTES);   // [2][128][PW]
     constexpr int NDG = tc_decode_groups(BN);            // groups of decoder warps
     // per decoder group: planes [kw*32][PWS], iz_stage [PW*32][kw], ip_stage [128][kw]
-    const int dgroup_words = g.kw * 32 * PWS + PW * 32 * g.kw + TC_BM * g.kw;
+    const int ikw = DW ? gi.kw : g.kw;                   // index words per factor row / column
+    const int dgroup_words = ikw * 32 * PWS + PW * 32 * ikw + TC_BM * ikw;
     const int dgrp = warp_of_thread_decoder_group(threadIdx.x);
     uint32_t *planes = row_bits + 2 * TC_BM * PW + dgrp * dgroup_words;
-    uint32_t *iz_stage = planes + g.kw * 32 * PWS;
-    uint32_t *ip_stage = iz_stage + PW * 32 * g.kw;
+    uint32_t *iz_stage = planes + ikw * 32 * PWS;
+    uint32_t *ip_stage = iz_stage + PW * 32 * ikw;
     uint8_t *epi_stage = reinterpret_cast<uint8_t *>(row_bits + 2 * TC_BM * PW + NDG * dgroup_words);   // PERSIST: 1 KB per pruning warp
     TcCtl *ctl = reinterpret_cast<TcCtl *>(epi_stage + (PERSIST ? TC_MASK_WARPS * 1024 : 0));
     volatile int *abort_flag = &ctl->abort_flag;
@@ -340,9 +345,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     // Long-latency requests first: the decoder warps ask for the factor words of their first panel, one
     // thread warms the TMA descriptors; both overlap the barrier and tensor-memory set-up below.
     {
-        const int npanels0 = (nkb + KBP - 1) / KBP;      // group g starts with panel g (of the block's first tiles)
+        const int npanels0 = DW ? BN / 256 : (nkb + KBP - 1) / KBP;   // group g starts with panel g (of the block's first tiles)
         if (warp >= 2 + TC_MASK_WARPS && dgrp < my_tiles * npanels0)
-            stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + (dgrp % npanels0) * KBP) * TC_BK,
+            stage_panel_factors(DW ? gi : g, rk, ip, iz, iz_stage, ip_stage, PW * 32,
+                                DW ? tile_b0(dgrp / npanels0) + (dgrp % npanels0) * 256 : (kb_begin + (dgrp % npanels0) * KBP) * TC_BK,
                                 tile_o0(dgrp / npanels0),
                                 (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1), TC_DECODE_WARPS * 32);
     }
@@ -466,13 +472,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         const int dt = (threadIdx.x - (2 + TC_MASK_WARPS) * 32) & (TC_DECODE_WARPS * 32 - 1);   // 0..127: row of the block this thread decodes
         const int dw = dt >> 5;                         // decoder warp 0..3
         const int bit_col = column_of_bit(lane);        // column (0..31) this lane stands for in a transpose
-        const int npanels = (nkb + KBP - 1) / KBP;
+        const Geo &gx = DW ? gi : g;                   // the layout the index is decoded from
+        const int npanels = DW ? BN / 256 : (nkb + KBP - 1) / KBP;
 
         // panels are counted across the block's tiles: panel PG is panel PG % npanels of tile PG / npanels
         auto stage_factors = [&](int PG) {
             if (PG < my_tiles * npanels) {
                 const int n2 = PG / npanels, P2 = PG - n2 * npanels;
-                stage_panel_factors(g, rk, ip, iz, iz_stage, ip_stage, PW * 32, (kb_begin + P2 * KBP) * TC_BK, tile_o0(n2), dt, TC_DECODE_WARPS * 32);
+                stage_panel_factors(gx, rk, ip, iz, iz_stage, ip_stage, PW * 32, DW ? tile_b0(n2) + P2 * 256 : (kb_begin + P2 * KBP) * TC_BK, tile_o0(n2), dt, TC_DECODE_WARPS * 32);
             }
         };
 
@@ -489,16 +496,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         for (int PG = dgrp; PG < my_tiles * npanels && ok; PG += NDG) {
             const int tile_n = PG / npanels, P = PG - tile_n * npanels;
             const int o0 = tile_o0(tile_n);
-            const int tr = o0 / g.tm;                   // the 128 rows lie in one tile row
-            const int i0 = o0 - tr * g.tm;              // first row of the block inside its tile
-            const bool row_ok = o0 + dt < g.rows && i0 + dt < g.tm;
+            const int tr = o0 / gx.tm;                   // the 128 rows lie in one tile row
+            const int i0 = o0 - tr * gx.tm;              // first row of the block inside its tile
+            const bool row_ok = o0 + dt < gx.rows && i0 + dt < gx.tm;
             const int buf = PG & 1;
             uint32_t *rb_buf = row_bits + buf * (TC_BM * PW);
-            const int c0 = (kb_begin + P * KBP) * TC_BK;
+            const int c0 = DW ? tile_b0(tile_n) + P * 256 : (kb_begin + P * KBP) * TC_BK;
             // rank of the panel's tile (the layout's, or the tile's own in a ranked layout)
-            int kp = g.k, kwp = g.kw;
+            int kp = gx.k, kwp = gx.kw;
             if (rk.ranks) {
-                kp = __ldg(rk.ranks + (size_t)min(tr, g.gr - 1) * g.ts_r + (size_t)(min(c0, g.cols - 1) / g.tn) * g.ts_c);
+                kp = __ldg(rk.ranks + (size_t)min(tr, gx.gr - 1) * gx.ts_r + (size_t)(min(c0, gx.cols - 1) / gx.tn) * gx.ts_c);
                 kwp = (kp + 31) >> 5;
             }
             const uint32_t tail = tail_mask(kp);
@@ -514,7 +521,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 for (int t = 0; t < 4; ++t) {
                     const int pi = dw + TC_DECODE_WARPS * (n0 + t);
                     const int lb = pi / PW, col = (pi % PW) * 32 + bit_col;
-                    z[t] = (pi < npairs && c0 + col < g.cols) ? iz_stage[col * kwp + lb] : 0u;
+                    z[t] = (pi < npairs && c0 + col < gx.cols) ? iz_stage[col * kwp + lb] : 0u;
                     if (lb == kwp - 1) z[t] &= tail;
                 }
                 warp_transpose32_x4(z, lane);
@@ -590,6 +597,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         for (int tile_n = 0; tile_n < my_tiles && ok; ++tile_n) {
         const int b0 = tile_b0(tile_n), o0 = tile_o0(tile_n);
         for (int it = 0; it < nkb && ok; ++it) {
+            if (DW) {                                    // nothing is pruned inside this contraction: pass the stage on
+                ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
+                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->masked[s]);
+                if (++s == stages) { s = 0; full_parity ^= 1; }
+                continue;
+            }
             const int buf = P & 1;
             if (kp == 0) {                               // first K block of a panel: its index bits must be there
                 ok = mbar_wait(&ctl->bits_ready[buf], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
@@ -623,10 +638,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             if (++s == stages) { s = 0; full_parity ^= 1; }
             if (++kp == KBP) { kp = 0; ++P; }
         }
-        if (kp != 0) { kp = 0; ++P; }                    // a tile's last panel may be short
+        if (!DW && kp != 0) { kp = 0; ++P; }             // a tile's last panel may be short
 
         // ------------------------------------------------------------- epilogue (same warps)
         if (ok) ok = mbar_wait(&ctl->accum, (uint32_t)(tile_n & 1), abort_flag, status, DEV_TIMEOUT_ACCUM);
+        if (ok && DW) {                                  // the index bits of the tile's two 256-column panels
+            ok = mbar_wait(&ctl->bits_ready[0], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
+            if (ok) ok = mbar_wait(&ctl->bits_ready[1], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
+        }
         if (ok && PERSIST) {
             // The operand stages already belong to the next tile: every warp moves its 32 output features x 16
             // (fp32: 8) batch columns through 1 KB of its own and stores 16-byte pieces, 64 (128) bytes of a row of Y
@@ -642,6 +661,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 uint32_t v[16];
                 tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)cl, v);
                 tmem_ld_wait();
+                if (DW) {
+                    // row quad*32+lane of the block, columns cl .. cl+15: panel cl/256, word (cl%256)/32; column e of a
+                    // word sits at bit 8 (e%4) + 7 - e/4 (the order the decoders write)
+                    const uint32_t wbits = row_bits[(cl >> 8) * (TC_BM * PW) + (quad * 32 + lane) * PW + ((cl & 255) >> 5)];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int e = (cl & 31) + j;
+                        if (!((wbits >> (8 * (e & 3) + 7 - (e >> 2))) & 1u)) v[j] = 0u;
+                    }
+                }
                 if (!out32) {
                     uint16_t *s16 = reinterpret_cast<uint16_t *>(st);
 #pragma unroll
@@ -685,7 +714,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             if (lane == 0) {
                 if (rank == 0) mbar_arrive(&ctl->tmem_free);
                 else mbar_arrive_remote(&ctl->tmem_free, 0);
+                if (DW) { mbar_arrive(&ctl->bits_free[0]); mbar_arrive(&ctl->bits_free[1]); }   // both index panels are used up
             }
+            if (DW) P += 2;
         }
         if (ok && !PERSIST) {
             tc_fence_after();
@@ -946,11 +977,12 @@ static int device_sm_count(int *dev_out)
     return sm_count;
 }
 
-template <int BN, int PW, bool PAIR, bool PERSIST>
+template <int BN, int PW, bool PAIR, bool PERSIST, bool DW = false>
 static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const uint16_t *W, const uint32_t *ip,
                              const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype,
-                             cudaStream_t s, float *partials, const TileRanks &rk)
+                             cudaStream_t s, float *partials, const TileRanks &rk, const Geo *index_geo = nullptr)
 {
+    const Geo gi = index_geo ? *index_geo : g;
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) { note_cuda_error(-1); return LRBI_ERR_CUDA; }
     CUtensorMap map;
@@ -970,7 +1002,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
-    auto kern = gemm_tc_kernel<BN, PW, PAIR, PERSIST>;
+    auto kern = gemm_tc_kernel<BN, PW, PAIR, PERSIST, DW>;
     {
         // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the function
         static bool attr_done[LRBI_MAX_DEVICES] = {false};
@@ -997,7 +1029,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int *status = device_status_ptr();
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, rk, ip, iz, batch, Y, y_dtype, partials, plan.kb_per_split, plan.stages, status);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, map, wmap, g, gi, rk, ip, iz, batch, Y, y_dtype, partials, plan.kb_per_split, plan.stages, status);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
@@ -1049,6 +1081,27 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
                            const uint16_t *X, int batch, void *Y, int y_dtype, cudaStream_t s, int force, const TileRanks *ranks)
 {
     return run_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, nullptr, 0, force, ranks);
+}
+
+// dW = (dY^T X) .* Ia on the persistent pair kernel: `g` describes the contraction (rows = cols of the layer, read from
+// Xt [layer cols][batch]; reduction over the batch; "batch" = rows of the layer, read from dYt [layer rows][batch]), `gi`
+// the index as the output tile sees it (the layer's layout transposed).  Returns LRBI_ERR_UNSUPPORTED when the shape
+// does not run on that kernel (the caller then takes another route).
+lrbi_status launch_gemm_tc_dw(const Geo &g, const Geo &gi, const uint16_t *Xt, const uint32_t *ip_t, const uint32_t *iz_t,
+                              const uint16_t *dYt, int out_rows, void *dW, int dtype, cudaStream_t s)
+{
+    if (!gemm_tc_supported(g, out_rows) || gi.k > TC_MAX_RANK) return LRBI_ERR_UNSUPPORTED;
+    if (!(gi.gr == 1 || (gi.tm % TC_BM) == 0) || !(gi.gc == 1 || (gi.tn % 256) == 0)) return LRBI_ERR_UNSUPPORTED;
+    int dev = -1;
+    const int sm_count = device_sm_count(&dev);
+    if (dev < 0) return LRBI_ERR_CUDA;
+    Geo gs = g;                                          // shared memory is sized for the index's rank
+    gs.k = gi.k; gs.kw = gi.kw;
+    TcPlan plan;
+    if (!make_tc_plan(gs, out_rows, sm_count, 2, &plan) || !plan.persist || plan.pw != 8) return LRBI_ERR_UNSUPPORTED;
+    if (!device_status_ptr()) return LRBI_ERR_CUDA;
+    const TileRanks none = {nullptr, nullptr, nullptr};
+    return launch_tc<512, 8, true, true, true>(gs, plan, dev, Xt, ip_t, iz_t, dYt, out_rows, dW, dtype, s, nullptr, none, &gi);
 }
 
 bool gemm_tc_plan(const Geo &g, int batch, int force, lrbi_gemm_plan *out)
