@@ -230,7 +230,7 @@ def kernel_label(B, layer, batch):
         return "decode"
     if batch < 0:
         return {-1: "index_cost", -2: "backward dX (forward kernel on the transposed layer)",
-                -3: "backward dW (2 transposes + tensor-core product + index applied in place)",
+                -3: "backward dW (2 transposes + persistent pair kernel, index applied in the epilogue)",
                 -4: "nmf, one multiplicative update of Mz and Mp (fp32 CUDA cores)"}[batch]
     plan = B.masked_gemm_plan(layer, batch)
     name = B.ALGO_NAMES[plan.algo]

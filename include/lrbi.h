@@ -292,8 +292,9 @@ LRBI_API lrbi_status lrbi_nmf_update(const lrbi_layout *layout, const uint16_t *
  * lrbi_masked_gemm_dw   dY [batch][rows], X [batch][cols] -> dW [rows][cols].  `workspace` is DEVICE memory of at least
  *       lrbi_masked_gemm_dw_workspace(layout, batch) bytes, 16-byte aligned, owned by the caller, scratch for the
  *       call (transposed copies of dY and X): the contraction runs on the tensor-core kernel with nothing pruned
- *       inside it, and the index, decoded on the fly and never stored, is then applied to dW in place.  batch % 8 != 0
- *       or a NULL workspace falls back to a slow one-thread-per-weight kernel.
+ *       inside it, and the index, decoded on the fly and never stored, is applied as dW is written (large aligned
+ *       shapes) or to dW in place afterwards.  batch % 8 != 0 or a NULL workspace falls back to a slow
+ *       one-thread-per-weight kernel.
  * lrbi_transpose_bf16   dst [cols][rows] = transpose of src [rows][cols] (bf16 bit patterns; dst must not overlap src).
  */
 LRBI_API lrbi_status lrbi_transpose_bf16(const uint16_t *src, int32_t rows, int32_t cols, uint16_t *dst, void *stream);

@@ -5,9 +5,11 @@
 //   dX   is the forward product of the TRANSPOSED layer: weights W^T (the caller keeps that copy), factors swapped
 //        (the row words of Ip are the column words of Ip^T and the other way round, so the packed arrays are used as
 //        they are, with the tile grid walked column-major);
-//   dW   is the forward product with X^T in the place of the weights and dY^T as the activations, with an index of
-//        rank one whose bits are all set (nothing pruned inside the contraction), written to dW; the index of the
-//        layer is then applied to dW in place by apply_index (decoded on the fly from bit-planes, never stored).
+//   dW   is the product with X^T in the place of the weights and dY^T as the activations, on the persistent pair
+//        kernel in its DW mode: nothing is pruned inside the contraction, the index of every output tile is decoded
+//        from the layer's factors (seen through the transposed layout) while the tile accumulates, and the epilogue
+//        writes zeros where Ia = 0.  Shapes that kernel does not take run the same product with an index of rank
+//        one whose bits are all set, followed by apply_index on dW in place.
 // This file holds the helper kernels: the bf16 transpose, the in-place application of the index, a filler, and a
 // slow any-shape dW.
 #include "lrbi_common.cuh"
@@ -29,11 +31,41 @@ transpose_bf16_kernel(const uint16_t *__restrict__ src, int rows, int cols, uint
         if (c0 + c < cols && r0 + tx < rows) dst[(size_t)(c0 + c) * rows + r0 + tx] = tile[tx][c];
 }
 
+// The same with 16-byte accesses on both sides (rows % 8 == 0, cols % 8 == 0): a thread reads 8 consecutive values of
+// a row, and writes 8 consecutive values of a row of the result gathered from a column of the tile.
+__global__ void __launch_bounds__(256)
+transpose_bf16_vec_kernel(const uint16_t *__restrict__ src, int rows, int cols, uint16_t *__restrict__ dst)
+{
+    __shared__ uint16_t tile[64][64 + 2];
+    const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int idx = threadIdx.x + 256 * u, r = idx >> 3, cs = (idx & 7) * 8;     // 64 rows x 8 pieces of 8
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r0 + r < rows && c0 + cs < cols) v = *reinterpret_cast<const uint4 *>(src + (size_t)(r0 + r) * cols + c0 + cs);
+        uint32_t *t32 = reinterpret_cast<uint32_t *>(&tile[r][cs]);                   // row pitch 132 bytes: 4-byte aligned
+        t32[0] = v.x; t32[1] = v.y; t32[2] = v.z; t32[3] = v.w;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int idx = threadIdx.x + 256 * u, c = idx >> 3, rs = (idx & 7) * 8;      // 64 result rows x 8 pieces of 8
+        if (c0 + c < cols && r0 + rs < rows) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) w[e] = (uint32_t)tile[rs + 2 * e][c] | ((uint32_t)tile[rs + 2 * e + 1][c] << 16);
+            *reinterpret_cast<uint4 *>(dst + (size_t)(c0 + c) * rows + r0 + rs) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
 lrbi_status launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst, cudaStream_t s)
 {
     dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
     if (grid.y > 65535) return LRBI_ERR_UNSUPPORTED;
-    transpose_bf16_kernel<<<grid, 256, 0, s>>>(src, rows, cols, dst);
+    const bool vec = (rows % 8) == 0 && (cols % 8) == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0;
+    if (vec) transpose_bf16_vec_kernel<<<grid, 256, 0, s>>>(src, rows, cols, dst);
+    else transpose_bf16_kernel<<<grid, 256, 0, s>>>(src, rows, cols, dst);
     count_launch();
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }

@@ -25,7 +25,7 @@ def rel_fro(got, want):
 def test_transpose_is_exact():
     b = _b()
     rng = np.random.default_rng(1)
-    for rows, cols in [(1, 1), (5, 70), (64, 64), (130, 257), (1000, 24)]:
+    for rows, cols in [(1, 1), (5, 70), (64, 64), (130, 257), (1000, 24), (72, 136), (512, 1032), (8, 8)]:
         a = rng.integers(0, 2**16, (rows, cols), dtype=np.uint16)
         got = b.lrbi_transpose_bf16(b.to_device_bf16(a)).view(torch.int16).cpu().numpy().view(np.uint16)
         assert (got == a.T).all()
