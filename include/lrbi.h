@@ -101,7 +101,8 @@ enum {
     /* The next two force an instantiation that LRBI_ALGO_TENSOR otherwise picks from the problem size
        (any shape LRBI_ALGO_TENSOR covers; small problems just leave most of a tile empty). */
     LRBI_ALGO_TENSOR_PAIR = 8,  /* tcgen05 CTA pairs (cta_group::2), 256 rows x 256 batch rows per pair  */
-    LRBI_ALGO_TENSOR_PAIR2 = 9  /* CTA pairs with two accumulators: 256 rows x 512 batch rows per pair   */
+    LRBI_ALGO_TENSOR_PAIR2 = 9, /* CTA pairs with two accumulators: 256 rows x 512 batch rows per pair   */
+    LRBI_ALGO_TENSOR_PAIR192 = 10 /* CTA pairs, one accumulator of 192 batch rows (few rows, long batch)   */
 };
 
 /* Element counts of the packed arrays for a layout (0 if the layout is invalid). */
@@ -133,7 +134,7 @@ LRBI_API lrbi_status lrbi_decode_mask(const lrbi_layout *layout, const uint32_t 
  *   X      device, bf16 bit patterns, [batch][cols] row-major
  *   Y      device, [batch][rows] row-major, bf16 (round to nearest even) or fp32 per y_dtype
  *   algo   LRBI_ALGO_AUTO, _GENERIC, _GEMV (batch <= 8), _STREAM (batch <= 32), _TENSOR, _TENSOR_PAIR or
- *          _TENSOR_PAIR2; a kernel that does not
+ *          _TENSOR_PAIR2 / _TENSOR_PAIR192; a kernel that does not
  *          cover the shape returns LRBI_ERR_UNSUPPORTED and launches nothing.
  * The tensor-core path may split the reduction over several thread blocks; it then keeps
  * fp32 partial sums in a library-owned device buffer that grows (cudaMalloc) on the first
@@ -287,7 +288,7 @@ LRBI_API lrbi_status lrbi_nmf_update(const lrbi_layout *layout, const uint16_t *
  * lrbi_masked_gemm_dx   needs the weights TRANSPOSED: Wt [cols][rows] bf16 (keep that copy beside W and refresh it with
  *       lrbi_transpose_bf16 when W changes).  It is the forward product of the transposed layer, so it runs on the same
  *       kernels: the packed factors are used as they are (a row word of Ip is a column word of Ip^T).  algo:
- *       LRBI_ALGO_AUTO, _GENERIC or _TENSOR / _TENSOR_PAIR / _TENSOR_PAIR2 (tensor-core shapes: rows % 8 == 0, and
+ *       LRBI_ALGO_AUTO, _GENERIC or _TENSOR / _TENSOR_PAIR / _TENSOR_PAIR2 / _TENSOR_PAIR192 (tensor-core shapes: rows % 8 == 0, and
  *       tile_cols % 128 == 0 and tile_rows % 64 == 0 unless the grid has one tile in that direction).
  * lrbi_masked_gemm_dw   dY [batch][rows], X [batch][cols] -> dW [rows][cols].  `workspace` is DEVICE memory of at least
  *       lrbi_masked_gemm_dw_workspace(layout, batch) bytes, 16-byte aligned, owned by the caller, scratch for the

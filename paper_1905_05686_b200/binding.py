@@ -18,8 +18,8 @@ from .synth import Layer
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblrbi.so")
 
-ALGO_AUTO, ALGO_GENERIC, ALGO_GEMV, ALGO_TENSOR, ALGO_DECODE_BALLOT, ALGO_DECODE_PLANES, ALGO_DECODE_PLANES_WIDE, ALGO_STREAM, ALGO_TENSOR_PAIR, ALGO_TENSOR_PAIR2 = range(10)
-ALGO_NAMES = {0: "auto", 1: "generic", 2: "gemv", 3: "tensor", 4: "decode_ballot", 5: "decode_planes", 6: "decode_planes_wide", 7: "stream", 8: "tensor_pair", 9: "tensor_pair2"}
+ALGO_AUTO, ALGO_GENERIC, ALGO_GEMV, ALGO_TENSOR, ALGO_DECODE_BALLOT, ALGO_DECODE_PLANES, ALGO_DECODE_PLANES_WIDE, ALGO_STREAM, ALGO_TENSOR_PAIR, ALGO_TENSOR_PAIR2, ALGO_TENSOR_PAIR192 = range(11)
+ALGO_NAMES = {0: "auto", 1: "generic", 2: "gemv", 3: "tensor", 4: "decode_ballot", 5: "decode_planes", 6: "decode_planes_wide", 7: "stream", 8: "tensor_pair", 9: "tensor_pair2", 10: "tensor_pair192"}
 Y_BF16, Y_F32 = 0, 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(6)
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024

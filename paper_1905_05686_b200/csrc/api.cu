@@ -151,6 +151,7 @@ lrbi_status lrbi_masked_gemm(const lrbi_layout *layout, const uint16_t *W, const
     case LRBI_ALGO_TENSOR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s);
     case LRBI_ALGO_TENSOR_PAIR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 1);
     case LRBI_ALGO_TENSOR_PAIR2: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 2);
+    case LRBI_ALGO_TENSOR_PAIR192: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 3);
     default: return LRBI_ERR_INVALID_ARG;
     }
 }
@@ -223,6 +224,7 @@ lrbi_status lrbi_masked_gemm_ranked(const lrbi_layout *layout, const lrbi_tile_r
     case LRBI_ALGO_TENSOR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 0, &rk);
     case LRBI_ALGO_TENSOR_PAIR: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 1, &rk);
     case LRBI_ALGO_TENSOR_PAIR2: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 2, &rk);
+    case LRBI_ALGO_TENSOR_PAIR192: return launch_gemm_tc(g, W, ip, iz, X, batch, Y, y_dtype, s, 3, &rk);
     default: return LRBI_ERR_INVALID_ARG;
     }
 }
@@ -278,6 +280,7 @@ lrbi_status lrbi_masked_gemm_dx(const lrbi_layout *layout, const uint16_t *Wt, c
     case LRBI_ALGO_TENSOR: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 0);
     case LRBI_ALGO_TENSOR_PAIR: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 1);
     case LRBI_ALGO_TENSOR_PAIR2: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 2);
+    case LRBI_ALGO_TENSOR_PAIR192: return launch_gemm_tc(t, Wt, iz, ip, dY, batch, dX, dx_dtype, s, 3);
     default: return LRBI_ERR_INVALID_ARG;
     }
 }
@@ -373,6 +376,7 @@ lrbi_status lrbi_masked_gemm_plan(const lrbi_layout *layout, int32_t batch, int3
     case LRBI_ALGO_TENSOR: return gemm_tc_plan(g, batch, 0, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
     case LRBI_ALGO_TENSOR_PAIR: return gemm_tc_plan(g, batch, 1, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
     case LRBI_ALGO_TENSOR_PAIR2: return gemm_tc_plan(g, batch, 2, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
+    case LRBI_ALGO_TENSOR_PAIR192: return gemm_tc_plan(g, batch, 3, plan) ? LRBI_OK : LRBI_ERR_UNSUPPORTED;
     default: return LRBI_ERR_INVALID_ARG;
     }
 }

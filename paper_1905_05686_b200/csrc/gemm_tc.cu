@@ -20,10 +20,10 @@
 //               planes selected by the set bits of that row's Ip word.  That is Eq. 3 evaluated 32
 //               columns per bitwise instruction; the result, the decoded index of the 128 x panel
 //               block, stays bit-packed in shared memory (double buffered) and goes nowhere else.
-//   warps 2-9   pruning warps.  A thread owns four 16-byte chunks of one row of the 128 x 64 block.
-//               When the stage's copies have landed it reads its chunks from the A stage, expands
-//               its 32 index bits to bf16 AND-masks (a shift puts four bits on the sign positions of
-//               the four bytes, prmt replicates each sign over a 16-bit half), zeroes pruned
+//   warps 2-9   pruning warps, two sets of four that take alternate K blocks.  A thread owns one row (eight
+//               16-byte chunks) of the 128 x 64 block.  When the stage's copies have landed it reads its chunks
+//               from the A stage, expands its 64 index bits to bf16 AND-masks (a shift puts four bits on the sign
+//               positions of the four bytes, prmt replicates each sign over a 16-bit half), zeroes pruned
 //               weights and writes the chunks back in place.  The writes are made visible to the
 //               tensor core with fence.proxy.async before the stage's "masked" barrier is signalled.
 //               No pruning warp ever waits on global memory.  After the last K block the same warps
@@ -47,9 +47,9 @@ constexpr int TC_BK = 64;                  // columns per stage: 64 bf16 = one 1
 constexpr int TC_A_STAGE_BYTES = TC_BM * TC_BK * 2;
 constexpr int TC_MASK_WARPS = 8;           // warps 2-9: prune the W tile of each stage, then run the epilogue
 constexpr int TC_DECODE_WARPS = 4;         // warps 10-13: decode the index one panel ahead
-// Two-accumulator blocks (BN = 512) run a second group of decoder warps (14-17): group g decodes the panels
+// Two-accumulator blocks (BN = 512) and the 192-column pairs run a second group of decoder warps (14-17): group g decodes the panels
 // with P % 2 == g into index buffer g, so a panel may take two panels' worth of pruning time.
-__host__ __device__ constexpr int tc_decode_groups(int bn) { return bn > 256 ? 2 : 1; }
+__host__ __device__ constexpr int tc_decode_groups(int bn) { return (bn > 256 || bn == 192) ? 2 : 1; }
 __host__ __device__ constexpr int tc_threads(int bn) { return TC_THREADS + (tc_decode_groups(bn) - 1) * TC_DECODE_WARPS * 32; }
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols)
 {
@@ -84,10 +84,12 @@ __device__ __forceinline__ uint32_t cluster_ctarank()
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync_all()
 {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    cluster_arrive();
+    cluster_wait();
 }
 __device__ __forceinline__ void tmem_alloc2(uint32_t *dst_smem, uint32_t ncols)
 {
@@ -221,7 +223,6 @@ struct TcCtl {
     uint64_t empty[8];       // the MMAs that read the stage have completed
     uint64_t accum;
     uint64_t tmem_free;      // PERSIST: tensor memory may be overwritten by the next tile's MMAs
-    uint64_t epi;            // the eight pruning warps meet here before the epilogue's copy-out
     uint64_t bits_ready[2];  // decoders -> pruners: the index bits of a panel are in buffer b
     uint64_t bits_free[2];   // pruners -> decoders: buffer b may be overwritten
     uint64_t dsync[2];       // the four warps of a decoder group meet here twice per panel
@@ -282,7 +283,7 @@ __device__ __forceinline__ int warp_of_thread_decoder_group(unsigned tid)
 // output sees it (rows = rows of the output tile, columns = its batch axis), the decoders decode the two 256-column
 // panels of each output tile from it, and the epilogue zeroes the pruned outputs as it stores them.
 template <int BN, int PW, bool PAIR, bool PERSIST, bool DW>
-__global__ void __launch_bounds__(tc_threads(BN), BN > 256 ? 1 : 2)
+__global__ void __launch_bounds__(tc_threads(BN), (BN > 256 || BN == 192) ? 1 : 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g, Geo gi, TileRanks rk,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
                void *__restrict__ Y, int y_dtype, float *__restrict__ partials, int kb_per_split,
@@ -291,15 +292,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     extern __shared__ __align__(1024) uint8_t smem[];    // swizzled operand stages need 1024-byte alignment
     constexpr int B_ROWS = PAIR ? BN / 2 : BN;          // rows of X this CTA loads per stage
     constexpr int B_STAGE_BYTES = B_ROWS * TC_BK * 2;
-    constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    constexpr int TMEM_COLS = BN < 32 ? 32 : BN == 192 ? 256 : BN;   // a power of two
     // Pair mode, BN = 512: two accumulators of 256 batch columns fill the 512 columns of tensor memory.
     // A pruned W stage then feeds two MMAs, so decode and pruning are amortised over twice the tensor work.
     // Accumulator a covers batch rows b0 + 256 a ...; CTA `rank` loads the 128 rows b0 + 256 a + 128 rank ...
     // of it as box a of its B stage.
-    constexpr int NACC = PAIR ? BN / 256 : 1;
-    constexpr int XBOX_ROWS = PAIR ? 128 : BN;          // rows of one TMA box of X
-    constexpr int MMA_N = PAIR ? 256 : BN;
-    static_assert(!PAIR || BN == 256 || BN == 512, "pair mode: one or two 256-column accumulators");
+    // BN = 192: one accumulator of 192 columns, 96 rows of X per CTA (a tile width that puts layers with few rows
+    // and a long batch on more of the chip's SMs: 12544 batch rows make 66 tiles of 192 against 25 of 512).
+    constexpr int NACC = PAIR && BN > 256 ? BN / 256 : 1;
+    constexpr int XBOX_ROWS = PAIR ? (BN < 256 ? BN / 2 : 128) : BN;   // rows of one TMA box of X
+    constexpr int MMA_N = PAIR ? (BN < 256 ? BN : 256) : BN;
+    static_assert(!PAIR || BN == 192 || BN == 256 || BN == 512, "pair mode: one accumulator of 192 or 256 columns, or two of 256");
+    static_assert(!PERSIST || BN == 512, "the persistent epilogue walks two 256-column accumulators");
     constexpr int KBP = PW / 2;                          // K blocks per panel
     uint8_t *a_base = smem;
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
@@ -356,22 +360,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&w_map) : "memory");
     }
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) {
-            mbar_init(&ctl->full[s], 1);
-            // leader of a pair: its stage is ready when its own eight pruning warps and the other CTA's relay have arrived
-            mbar_init(&ctl->masked[s], TC_MASK_WARPS + ((PAIR && rank == 0) ? 1 : 0));
-            mbar_init(&ctl->empty[s], 1);
-        }
-        mbar_init(&ctl->accum, 1);
-        mbar_init(&ctl->epi, TC_MASK_WARPS);
-        mbar_init(&ctl->tmem_free, 2 * TC_MASK_WARPS);   // PERSIST, leader: the pruning warps of both CTAs have drained tensor memory
-        for (int b = 0; b < 2; ++b) {
+    if (warp == 0) {                                     // one lane per stage, three more for the rest
+        if (lane < stages) {
+            mbar_init(&ctl->full[lane], 1);
+            // leader of a pair: its stage is ready when its own four pruning warps of the K block's set and the other CTA's relay have arrived
+            mbar_init(&ctl->masked[lane], TC_MASK_WARPS / 2 + ((PAIR && rank == 0) ? 1 : 0));   // one set of pruning warps per K block
+            mbar_init(&ctl->empty[lane], 1);
+        } else if (lane == 8) {
+            mbar_init(&ctl->accum, 1);
+            mbar_init(&ctl->tmem_free, 2 * TC_MASK_WARPS);   // PERSIST, leader: the pruning warps of both CTAs have drained tensor memory
+            ctl->abort_flag = 0;
+        } else if (lane == 9 || lane == 10) {
+            const int b = lane - 9;
             mbar_init(&ctl->bits_ready[b], TC_DECODE_WARPS);
             mbar_init(&ctl->bits_free[b], TC_MASK_WARPS);
+            mbar_init(&ctl->dsync[b], TC_DECODE_WARPS);
         }
-        for (int b = 0; b < 2; ++b) mbar_init(&ctl->dsync[b], TC_DECODE_WARPS);
-        ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -380,20 +384,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
-    if (PAIR) cluster_sync_all();                        // both CTAs' barriers exist before anyone signals across
+    // Both CTAs' barriers must exist before anyone signals across.  Everybody arrives at the cluster barrier now; the
+    // warp of the TMA producer waits only after its first round of copies is on its way (they touch this CTA alone).
+    if (PAIR) {
+        cluster_arrive();
+        if (warp != 0) cluster_wait();
+    }
     tc_fence_after();
     const uint32_t tmem_d = ctl->tmem_base;
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer (X tiles)
-        if (lane == 0) {
-            bool issued = false;
-            int s = 0;
-            uint32_t parity = 1;                        // a fresh barrier reports its "previous" phase complete
-            bool go = true;
-            for (int n = 0; n < my_tiles && go; ++n) {
-            const int b0 = tile_b0(n), o0 = tile_o0(n);
-            for (int it = 0; it < nkb; ++it) {
+        bool issued = false;
+        int s = 0;
+        uint32_t parity = 1;                            // a fresh barrier reports its "previous" phase complete
+        bool go = true;
+        const long long total = (long long)my_tiles * nkb;
+        auto issue = [&](long long q0, long long q1) {  // K blocks q0 .. q1-1, counted across the block's tiles
+            for (long long q = q0; q < q1 && go; ++q) {
+                const int n = (int)(q / nkb), it = (int)(q - (long long)n * nkb);
+                const int b0 = tile_b0(n), o0 = tile_o0(n);
                 if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) { go = false; break; }
                 mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES + TC_A_STAGE_BYTES);
                 tma_load_2d(a_base + s * TC_A_STAGE_BYTES, &w_map, &ctl->full[s], (kb_begin + it) * TC_BK, o0);
@@ -404,7 +414,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 issued = true;
                 if (++s == stages) { s = 0; parity ^= 1; }
             }
-            }
+        };
+        const long long first = total < stages ? total : stages;   // the ring's first round needs nobody else
+        if (lane == 0) issue(0, first);
+        __syncwarp();
+        if (PAIR) cluster_wait();
+        if (lane == 0) {
+            issue(first, total);
             if (*abort_flag && issued) {
                 // Abort path: copies already issued must land before this block's shared memory is
                 // given up.  Wait on elapsed cycles alone (bounded): about 2 ms, far beyond any copy
@@ -580,61 +596,69 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         // ------------------------------------------------------------- pruning warps
         const int mt = threadIdx.x - 64;                // 0..255
         const int mw = mt >> 5;                         // pruning warp 0..7
-        // Two lanes share a row: lane pair p of a warp owns row 8*(p/8) + 2*(p%4) + (p/4)%2 of the
-        // warp's 16 rows (so the eight lanes of one store phase fall on eight different swizzled
-        // chunk positions), and lane h of the pair owns the 16-byte chunks h, h+2, h+4, h+6 of the
-        // row's 128 bytes.
-        const int pr = lane >> 1;
-        const int r = mw * 16 + 8 * (pr >> 3) + 2 * (pr & 3) + ((pr >> 2) & 1);   // row of the 128-row block
-        const int h = lane & 1;
-        uint32_t epi_parity = 0;
+        // The warps form two sets of four that take alternate K blocks (set q: the blocks whose running number is
+        // q mod 2), so the wait - load - prune - store - fence - arrive chain of one K block overlaps the next
+        // block's: the chain is latency, not work, and one set alone was measured at half a microsecond per block.
+        // Inside a set a thread owns one row of the 128 (eight 16-byte chunks; the eight lanes of one access phase
+        // fall on eight different swizzled chunk positions).
+        const int set = mw >> 2;
+        const int r = (mw & 3) * 32 + lane;             // row of the 128-row block
 
         bool ok = true;
         int s = 0;                                       // stage of the current K block
         uint32_t full_parity = 0;
         int kp = 0;                                      // K block inside its panel
         int P = 0;                                       // panel index, counted across the block's tiles
+        int P_seen = -1;                                 // last panel whose index bits this warp has waited for
+        uint32_t G = 0;                                  // running number of the K block, across the block's tiles
+        auto panel_bits_ready = [&]() {                  // (every warp waits for every panel, also one it takes no block of:
+            if (P_seen != P) {                           //  its arrival below must not run ahead of the decoders)
+                ok = mbar_wait(&ctl->bits_ready[P & 1], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
+                P_seen = P;
+            }
+        };
         for (int tile_n = 0; tile_n < my_tiles && ok; ++tile_n) {
         const int b0 = tile_b0(tile_n), o0 = tile_o0(tile_n);
-        for (int it = 0; it < nkb && ok; ++it) {
+        for (int it = 0; it < nkb && ok; ++it, ++G) {
+            const bool mine = (G & 1u) == (uint32_t)set;
             if (DW) {                                    // nothing is pruned inside this contraction: pass the stage on
-                ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
-                if (!ok) break;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->masked[s]);
+                if (mine) {
+                    ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
+                    if (!ok) break;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->masked[s]);
+                }
                 if (++s == stages) { s = 0; full_parity ^= 1; }
                 continue;
             }
             const int buf = P & 1;
-            if (kp == 0) {                               // first K block of a panel: its index bits must be there
-                ok = mbar_wait(&ctl->bits_ready[buf], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
+            if (mine) {
+                panel_bits_ready();
                 if (!ok) break;
+                const uint2 bits = *reinterpret_cast<const uint2 *>(row_bits + buf * (TC_BM * PW) + r * PW + kp * 2);
+                // ---------------- prune the 64 weights of one row of the A stage, in place
+                ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
+                if (!ok) break;
+                uint8_t *a_row = a_base + s * TC_A_STAGE_BYTES + r * 128;
+                uint4 wv[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c)              // 128-byte swizzle: 16-byte chunk c of row r lives at chunk position c ^ (r % 8)
+                    wv[c] = *reinterpret_cast<const uint4 *>(a_row + ((c ^ (r & 7)) << 4));
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {            // chunk c: index word c / 4, chunk-in-word c % 4
+                    wv[c] = prune_chunk(wv[c], (c < 4) ? bits.x : bits.y, c & 3);
+                    *reinterpret_cast<uint4 *>(a_row + ((c ^ (r & 7)) << 4)) = wv[c];
+                }
+                fence_async_proxy();                     // generic-proxy stores -> visible to the MMA
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->masked[s]);
             }
-            const uint2 bits = *reinterpret_cast<const uint2 *>(row_bits + buf * (TC_BM * PW) + r * PW + kp * 2);
-            if (kp == KBP - 1 || it == nkb - 1) {        // last use of this buffer: hand it back to the decoders
+            if (kp == KBP - 1 || it == nkb - 1) {        // the panel ends: hand its buffer back to the decoders
+                panel_bits_ready();
+                if (!ok) break;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->bits_free[buf]);
             }
-            // ---------------- prune 32 weights of one row of the A stage, in place
-            ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
-            if (!ok) break;
-            uint8_t *a_row = a_base + s * TC_A_STAGE_BYTES + r * 128;
-            uint4 wv[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                // 128-byte swizzle: 16-byte chunk c of row r lives at chunk position c ^ (r % 8)
-                const int chunk = 2 * j + h;
-                wv[j] = *reinterpret_cast<const uint4 *>(a_row + ((chunk ^ (r & 7)) << 4));
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {                // chunk 2j+h: word (2j+h)/4, chunk-in-word (2j+h)%4
-                const int chunk = 2 * j + h;
-                wv[j] = prune_chunk(wv[j], (j < 2) ? bits.x : bits.y, chunk & 3);
-                *reinterpret_cast<uint4 *>(a_row + ((chunk ^ (r & 7)) << 4)) = wv[j];
-            }
-            fence_async_proxy();                         // generic-proxy stores -> visible to the MMA
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->masked[s]);
             if (++s == stages) { s = 0; full_parity ^= 1; }
             if (++kp == KBP) { kp = 0; ++P; }
         }
@@ -720,70 +744,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         }
         if (ok && !PERSIST) {
             tc_fence_after();
-            // All MMAs have completed, so the operand stages are free: reuse them to transpose the
-            // accumulator (lane = output feature) into rows of Y (contiguous output features).  The
-            // accumulator goes through in as few passes as the stage memory allows (all 256 columns at once
-            // for bf16 output in pair mode, halves for fp32).
+            // All MMAs have completed.  In tensor memory a lane is an output feature and a column a batch row, so the 32
+            // lanes of a warp hold 32 consecutive outputs of one row of Y: every column goes out as one 64-byte (fp32:
+            // 128-byte) warp store straight from the registers, whole sectors, no staging and no meeting of the warps.
             const bool out32 = partials != nullptr || y_dtype == LRBI_Y_F32;
-            const int esz = out32 ? 4 : 2;
             const int quad = warp & 3;                   // tensor-memory lanes this warp may read
-            const int half = mw >> 2;                    // which half of a pass's columns
-            const int ol = quad * 32 + lane;             // output feature inside the block
-            const int room = stages * (TC_A_STAGE_BYTES + B_STAGE_BYTES) / (TC_BM * esz);   // columns the stages can hold
-            int PASS = BN;                               // batch columns per pass: BN, BN/2, ... down to 32 (or BN if smaller)
-            while (PASS > 32 && PASS > room) PASS >>= 1;                                    // always a divisor of BN
-            const int COLS_PER_WARP = PASS / 2 < 16 ? 16 : PASS / 2;
-            const int NCHUNK = COLS_PER_WARP / 16;
+            const int half = mw >> 2;                    // which half of the tile's columns
+            constexpr int HC = BN >= 32 ? BN / 2 : BN;   // columns per warp (a 16-column tile: the first four warps only)
+            const int o = o0 + quad * 32 + lane;         // this lane's output feature
+            const bool o_ok = o < g.rows;
             uint8_t *dst_base = partials ? reinterpret_cast<uint8_t *>(partials + (long long)blockIdx.z * batch * g.rows)
                                          : reinterpret_cast<uint8_t *>(Y);
-            const int row_bytes = TC_BM * esz;           // one batch row of the block
-            const int chunks = row_bytes / 16;           // 16 (bf16) or 32 (fp32)
-            const int per16 = 16 / esz;                  // outputs per 16-byte chunk
-            const bool vec_ok = (g.rows % per16) == 0;   // rows of Y stay 16-byte aligned
-            auto meet = [&]() {                          // the eight warps meet (bounded wait)
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->epi);
-                ok = mbar_wait(&ctl->epi, epi_parity, abort_flag, status, DEV_TIMEOUT_ACCUM);
-                epi_parity ^= 1;
-            };
+            if (BN >= 32 || half == 0) {
 #pragma unroll 1
-            for (int pass0 = 0; pass0 < BN && ok; pass0 += PASS) {
-                if ((PASS >= 32) || half == 0) {
-#pragma unroll 1
-                    for (int ch = 0; ch < NCHUNK; ++ch) {
-                        const int cl = half * COLS_PER_WARP + ch * 16;       // column inside the pass
-                        uint32_t v[16];
-                        tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass0 + cl), v);
-                        tmem_ld_wait();
-                        if (out32) {
-                            float *st = reinterpret_cast<float *>(smem);
+                for (int ch = 0; ch < HC / 16; ++ch) {
+                    const int cl = half * HC + ch * 16;  // first batch column of the chunk inside the tile
+                    if (b0 + cl >= batch) break;         // (the whole warp) the rest of the tile lies outside the batch
+                    uint32_t v[16];
+                    tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)cl, v);
+                    tmem_ld_wait();
+                    const long long row0 = (long long)(b0 + cl) * g.rows + o;
+                    if (out32) {
+                        float *dst = reinterpret_cast<float *>(dst_base) + row0;
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) st[(cl + j) * TC_BM + ol] = __uint_as_float(v[j]);
-                        } else {
-                            uint16_t *st = reinterpret_cast<uint16_t *>(smem);
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) st[(cl + j) * TC_BM + ol] = f32_to_bf16_rne(__uint_as_float(v[j]));
-                        }
-                    }
-                }
-                meet();                                  // the pass is staged
-                if (!ok) break;
-                const int nb = min(PASS, batch - b0 - pass0);
-                for (int idx = mt; idx < nb * chunks; idx += TC_MASK_WARPS * 32) {
-                    const int bl = idx / chunks, cj = idx - bl * chunks;
-                    const int oc = o0 + cj * per16;      // first output feature of the chunk
-                    if (oc >= g.rows) continue;
-                    const uint8_t *src = smem + (size_t)bl * row_bytes + cj * 16;
-                    uint8_t *dst = dst_base + ((long long)(b0 + pass0 + bl) * g.rows + oc) * esz;
-                    if (vec_ok && oc + per16 <= g.rows) {
-                        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+                        for (int j = 0; j < 16; ++j)
+                            if (o_ok && b0 + cl + j < batch) dst[(long long)j * g.rows] = __uint_as_float(v[j]);
                     } else {
-                        const int n = min(per16, g.rows - oc);
-                        for (int e = 0; e < n * esz; e += 2)
-                            *reinterpret_cast<uint16_t *>(dst + e) = *reinterpret_cast<const uint16_t *>(src + e);
+                        uint16_t *dst = reinterpret_cast<uint16_t *>(dst_base) + row0;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (o_ok && b0 + cl + j < batch) dst[(long long)j * g.rows] = f32_to_bf16_rne(__uint_as_float(v[j]));
                     }
                 }
-                if (pass0 + PASS < BN) meet();           // staging may be overwritten by the next pass
             }
         }
         }                                                // the block's tiles
@@ -890,7 +882,7 @@ struct TcPlan {
 };
 
 // `force`: 0 = choose by shape; 1 = CTA pairs with one accumulator (256 batch columns per pair);
-// 2 = CTA pairs with two accumulators (512 batch columns per pair).
+// 2 = CTA pairs with two accumulators (512 batch columns per pair); 3 = CTA pairs with one accumulator of 192 columns.
 static bool make_tc_plan(const Geo &g, int batch, int sm_count, int force, TcPlan *out)
 {
     if (!gemm_tc_supported(g, batch)) return false;
@@ -901,7 +893,12 @@ static bool make_tc_plan(const Geo &g, int batch, int sm_count, int force, TcPla
     // batch rows, two accumulators whenever the batch has more than 256 rows.
     p.pair = force ? true : (batch > 128 && g.rows > TC_BM);
     p.bn = batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : 128;
-    if (p.pair) p.bn = force == 1 ? 256 : force == 2 ? 512 : (batch > 256 ? 512 : 256);
+    if (p.pair) p.bn = force == 1 ? 256 : force == 2 ? 512 : force == 3 ? 192 : (batch > 256 ? 512 : 256);
+    // Few rows and a long batch (a lowered convolution): tiles of 512 batch rows leave most SMs idle.  When the
+    // 192-row tiles fit the chip in one wave of pairs they win (measured, 256 x 2304 weights: 12544 batch rows
+    // 33.9 us against 48.1, 3136 rows 25.6 against 31.7; 300 x 1000 weights, 777 rows 19.4 against 25.4).
+    if (p.pair && force == 0 && batch > 256 &&
+        (long long)((batch + 191) / 192) * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) <= sm_count / 2) p.bn = 192;
     // index words per panel row: 256-column panels when every panel then lies inside one tile
     p.pw = (g.gc == 1 || (g.tn % 256) == 0) ? 8 : 2;
     const int nkb = (g.cols + TC_BK - 1) / TC_BK;
@@ -919,7 +916,7 @@ static bool make_tc_plan(const Geo &g, int batch, int sm_count, int force, TcPla
         // A lone block advances about one K block per microsecond (its ring of stages is bound by latency, not
         // by the tensor pipe), so cutting K pays when blocks are few -- as long as writing and re-reading the
         // fp32 partial sums (about 5 bytes per nanosecond) costs less than half of the time it saves.
-        const long long slots = (long long)sm_count * (p.bn == 512 ? 1 : 2);
+        const long long slots = (long long)sm_count * ((p.bn == 512 || p.bn == 192) ? 1 : 2);   // blocks resident at once
         if (tiles < slots) {
             int sp = (int)(slots / tiles);
             if (sp > nkb / 8) sp = nkb / 8;           // at least 8 K blocks per split
@@ -957,7 +954,8 @@ static bool make_tc_plan(const Geo &g, int batch, int sm_count, int force, TcPla
     const size_t per_stage = TC_A_STAGE_BYTES + b_stage;
     const size_t half_sm = 113 * 1024, whole_sm = 224 * 1024;
     int stages = (int)((half_sm - extras) / per_stage);
-    if (extras > half_sm || stages < 3) stages = (int)((whole_sm - extras) / per_stage);
+    // (a grid of no more blocks than SMs has an SM per block anyway: deeper rings for those)
+    if (extras > half_sm || stages < 3 || tiles * p.splits <= sm_count || p.bn == 192) stages = (int)((whole_sm - extras) / per_stage);
     if (stages > 6) stages = 6;
     if (stages < 2) return false;
     p.stages = stages;
@@ -988,7 +986,7 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.cols, (cuuint64_t)batch};
     const cuuint64_t strides[1] = {(cuuint64_t)g.cols * 2};
-    const cuuint32_t box[2] = {TC_BK, PAIR ? 128 : BN};
+    const cuuint32_t box[2] = {TC_BK, PAIR ? (BN < 256 ? BN / 2 : 128) : BN};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1069,6 +1067,7 @@ static lrbi_status run_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, c
     LRBI_TC_CASE(32, 8, false) LRBI_TC_CASE(32, 2, false)
     LRBI_TC_CASE(64, 8, false) LRBI_TC_CASE(64, 2, false)
     LRBI_TC_CASE(128, 8, false) LRBI_TC_CASE(128, 2, false)
+    LRBI_TC_CASE(192, 8, true) LRBI_TC_CASE(192, 2, true)
     LRBI_TC_CASE(256, 8, true) LRBI_TC_CASE(256, 2, true)
     LRBI_TC_CASE(512, 8, true) LRBI_TC_CASE(512, 2, true)
     if (plan.persist && plan.pw == 8) return launch_tc<512, 8, true, true>(g, plan, dev, W, ip, iz, X, batch, Y, y_dtype, s, partials, rk);

@@ -57,7 +57,7 @@ def test_masked_backward(shape):
     W, X, dY = b.to_device_bf16(Wb), b.to_device_bf16(Xb), b.to_device_bf16(dYb)
     Wt = b.lrbi_transpose_bf16(W)
     tc_ok = rows % 8 == 0 and (L.grid[1] == 1 or tn % 128 == 0) and (L.grid[0] == 1 or tm % 64 == 0)
-    algos = [b.ALGO_GENERIC, b.ALGO_AUTO] + ([b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2] if tc_ok else [])
+    algos = [b.ALGO_GENERIC, b.ALGO_AUTO] + ([b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2, b.ALGO_TENSOR_PAIR192] if tc_ok else [])
     for algo in algos:
         for dt, tol in ((torch.bfloat16, TOL), (torch.float32, TOL_F32)):
             got = b.lrbi_masked_gemm_dx(L, Wt, ip, iz, dY, dtype=dt, algo=algo).float().cpu().numpy().astype(np.float64)

@@ -290,8 +290,9 @@ def test_ffn_config_full():
 
 # ------------------------------------------------------------------------------------------------
 # CTA-pair instantiations of the tensor-core kernel (the ones large layers run on), with one accumulator
-# (256 batch rows per pair) and with two (512 batch rows per pair; the headline workload's kernel).  They
-# are forced through LRBI_ALGO_TENSOR_PAIR / _PAIR2 so that every shape below runs in both; the shapes are
+# (256 batch rows per pair, or 192: the tile of layers with few rows and a long batch) and with two (512 batch
+# rows per pair; the headline workload's kernel).  They are forced through LRBI_ALGO_TENSOR_PAIR / _PAIR192 /
+# _PAIR2 so that every shape below runs in all three; the shapes are
 # wide in the batch and thin in K (the oracle stays under a second each).
 # ------------------------------------------------------------------------------------------------
 PAIR_SHAPES = [
@@ -310,10 +311,10 @@ PAIR_SHAPES = [
 
 def _pair_algos():
     b = _b()
-    return [(b.ALGO_TENSOR_PAIR, 256), (b.ALGO_TENSOR_PAIR2, 512)]
+    return [(b.ALGO_TENSOR_PAIR, 256), (b.ALGO_TENSOR_PAIR2, 512), (b.ALGO_TENSOR_PAIR192, 192)]
 
 
-@pytest.mark.parametrize("width", [256, 512])
+@pytest.mark.parametrize("width", [192, 256, 512])
 @pytest.mark.parametrize("shape", PAIR_SHAPES, ids=lambda s: "x".join(map(str, s)))
 def test_cta_pair_kernel(shape, width):
     b = _b()
@@ -329,9 +330,14 @@ def test_cta_pair_kernel(shape, width):
     assert b.launch_count() - before == 2 * (1 if plan.k_splits == 1 else 2)
 
 
-def test_auto_choice_reaches_both_pair_instantiations():
-    """What LRBI_ALGO_TENSOR picks by itself: pairs above 128 batch rows, two accumulators above 256."""
+def test_auto_choice_reaches_every_pair_instantiation():
+    """What LRBI_ALGO_TENSOR picks by itself: pairs above 128 batch rows, two accumulators above 256, and 192-row
+    tiles when those fit the chip in one wave (few rows, long batch)."""
     b = _b()
+    L = synth.Layer("few", 256, 576, 128, 64, 16, 0.25, 0.05)
+    plan = b.masked_gemm_plan(L, 1500, b.ALGO_TENSOR)
+    assert plan.cta_pair == 1 and plan.batch_tile == 192
+    Case(L, 1500).check_full(b.ALGO_TENSOR)
     L = synth.Layer("pair", 1024, 512, 512, 256, 64, 0.25, 0.05)
     for batch, width in ((200, 256), (7200, 512)):
         plan = b.masked_gemm_plan(L, batch, b.ALGO_TENSOR)
@@ -344,7 +350,7 @@ def test_auto_choice_reaches_both_pair_instantiations():
     Case(L, 300).check_full(b.ALGO_TENSOR)
 
 
-@pytest.mark.parametrize("width", [256, 512])
+@pytest.mark.parametrize("width", [192, 256, 512])
 def test_cta_pair_kernel_one_hot_and_degenerate_masks(width):
     b = _b()
     algo = dict((w, a) for a, w in _pair_algos())[width]
@@ -386,7 +392,7 @@ def test_bits_beyond_rank_are_ignored_by_every_gemm_kernel(k):
     b = _b()
     L = synth.Layer("pad", 256, 512, 128, 128, k, 0.25, 0.05)
     garbage = np.uint32((0xFFFFFFFF << (k % 32)) & 0xFFFFFFFF)
-    for batch, algos in ((4, (b.ALGO_GENERIC, b.ALGO_GEMV, b.ALGO_STREAM)), (40, (b.ALGO_TENSOR,)), (300, (b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2))):
+    for batch, algos in ((4, (b.ALGO_GENERIC, b.ALGO_GEMV, b.ALGO_STREAM)), (40, (b.ALGO_TENSOR,)), (300, (b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2, b.ALGO_TENSOR_PAIR192))):
         c = Case(L, batch)
         want = c.oracle_full()
         ipw, izw = synth.pack_ip(c.Ip).reshape(-1, L.kw), synth.pack_iz(c.Iz).reshape(-1, L.kw)

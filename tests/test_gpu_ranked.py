@@ -69,7 +69,7 @@ def test_ranked_decode_and_product(shape):
         X = b.to_device_bf16(Xb)
         algos = [b.ALGO_GENERIC, b.ALGO_AUTO]
         if L.cols % 8 == 0 and (L.grid[0] == 1 or L.tile_rows % 128 == 0) and (L.grid[1] == 1 or L.tile_cols % 64 == 0):
-            algos += [b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2]
+            algos += [b.ALGO_TENSOR, b.ALGO_TENSOR_PAIR, b.ALGO_TENSOR_PAIR2, b.ALGO_TENSOR_PAIR192]
         for algo in algos:
             for dt, tol in ((torch.bfloat16, TOL), (torch.float32, TOL_F32)):
                 Y = b.lrbi_masked_gemm_ranked(L, rk, ipo, izo, W, ip, iz, X, y_dtype=dt, algo=algo)
