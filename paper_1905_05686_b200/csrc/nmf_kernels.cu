@@ -4,130 +4,289 @@
 // The paper leaves the solver to "an NMF library"; this is the update rule of the NMF reference it cites.
 // All arithmetic is fp32 on CUDA cores (the factors are real-valued and the iteration is sensitive to rounding; the
 // two large products per iteration are 4 k tm tn flops per tile, small against the layer's own GEMMs).
-//   nmf_gemm<0>   N1 = Mp^T |W|   (k x tn per tile)         nmf_gemm<1>   N2 = |W| Mz^T   (tm x k per tile)
+//   nmf_prod_z    N1 = Mp^T |W|   (k x tn per tile)         nmf_prod_p    N2 = |W| Mz^T   (tm x k per tile)
+//                 (a thread owns one output column / row and 32 rank values; |W| is read once per 32 rank values)
 //   nmf_gram      G  = Mp^T Mp  or  Mz Mz^T   (k x k per tile)
 //   nmf_update_z / nmf_update_p   the element-wise update with the k-term denominator
 #include "lrbi_common.cuh"
 
 namespace lrbi {
 
-constexpr int NG_T = 64;               // output tile of the product kernels
-constexpr int NG_K = 16;               // reduction step
+constexpr int NP_THREADS = 128;        // outputs of a product block: one column (prod_z) or row (prod_p) per thread.x
+constexpr int NP_GROUPS = 4;           // threads per output (thread.y): each takes a quarter of every slab of the reduction
+constexpr int NP_KC = 32;              // rank values per block: a thread keeps that many running sums in registers
+constexpr int NP_SLAB0 = 32;           // rows of the reduction staged per step, prod_z
+constexpr int NP_SLAB1 = 64;           // columns of the reduction staged per step, prod_p
 
 __device__ __forceinline__ float abs_bf16(uint16_t h) { return __uint_as_float(((uint32_t)h << 16) & 0x7FFF0000u); }
 
-// MODE 0: C[l][j] = sum_i P[i][l] |W[i][j]|   (rows of C: k, columns: tn, reduction: tm)
-// MODE 1: C[i][l] = sum_j |W[i][j]| Z[l][j]   (rows of C: tm, columns: k, reduction: tn)
-// grid = (column tiles, row tiles, layer tiles); 256 threads, 4 x 4 outputs each.
-template <int MODE>
-__global__ void __launch_bounds__(256)
-nmf_gemm_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__ F, float *__restrict__ C)
+// N1[l][j] = sum_i P[i][l] |W[i][j]|   (k x tn per tile; the reduction runs over the tile's rows).
+// grid = (ceil(tn / 128), layer tiles, ceil(k / 32)).  A thread owns column j and 32 values of l: |W[i][j]| comes
+// straight from device memory (consecutive threads, consecutive columns), the 32 values P[i][l] of a row are read
+// from shared memory by every thread alike (broadcast), 32 multiply-adds per weight.  Four threads share a column
+// (each takes a quarter of a slab's rows) and add their sums up through shared memory at the end.
+__device__ __forceinline__ void nmf_fold_groups(float (&acc)[NP_KC], float *red, int t, int q)
 {
-    __shared__ float As[NG_K][NG_T + 4], Bs[NG_K][NG_T + 4];
-    const int tile = blockIdx.z, tr = tile / g.gc, tc = tile - tr * g.gc;
-    const int k = g.k;
-    const int CM = MODE == 0 ? k : g.tm, CN = MODE == 0 ? g.tn : k, KR = MODE == 0 ? g.tm : g.tn;
-    const int m0 = blockIdx.y * NG_T, n0 = blockIdx.x * NG_T;
-    const uint16_t *Wt = W + (size_t)tr * g.tm * g.cols + (size_t)tc * g.tn;
+    for (int qq = 1; qq < NP_GROUPS; ++qq) {
+        __syncthreads();
+        if (q == qq) {
+#pragma unroll
+            for (int c = 0; c < NP_KC; ++c) red[c * NP_THREADS + t] = acc[c];
+        }
+        __syncthreads();
+        if (q == 0) {
+#pragma unroll
+            for (int c = 0; c < NP_KC; ++c) acc[c] += red[c * NP_THREADS + t];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(NP_THREADS * NP_GROUPS, 2)
+nmf_prod_z_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__ P, float *__restrict__ N1)
+{
+    __shared__ __align__(16) float Ps[NP_SLAB0][NP_KC];
+    __shared__ float red[NP_KC * NP_THREADS];
+    const int tile = blockIdx.y, tr = tile / g.gc, tc = tile - tr * g.gc, k = g.k, t = threadIdx.x, q = threadIdx.y;
+    const int tid = q * NP_THREADS + t;
+    constexpr int RQ = NP_SLAB0 / NP_GROUPS;            // rows of a slab per thread
+    const int j = blockIdx.x * NP_THREADS + t, l0 = blockIdx.z * NP_KC, kc = min(NP_KC, k - l0);
     const int wrows = min(g.tm, g.rows - tr * g.tm), wcols = min(g.tn, g.cols - tc * g.tn);   // part of the tile inside the matrix
-    const float *Ft = F + (size_t)tile * (MODE == 0 ? (size_t)g.tm * k : (size_t)k * g.tn);
-    float *Ct = C + (size_t)tile * CM * CN;
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-    float acc[4][4] = {};
-    for (int r0 = 0; r0 < KR; r0 += NG_K) {
-        for (int e = threadIdx.x; e < NG_K * NG_T; e += 256) {
-            if (MODE == 0) {
-                const int kk = e / NG_T, m = e - kk * NG_T;             // consecutive threads: consecutive l (contiguous in P)
-                const int i = r0 + kk, l = m0 + m;
-                As[kk][m] = (i < g.tm && l < k) ? Ft[(size_t)i * k + l] : 0.f;
-                const int j = n0 + m;                                    // and consecutive j (contiguous in W)
-                Bs[kk][m] = (i < wrows && j < wcols) ? abs_bf16(Wt[(size_t)i * g.cols + j]) : 0.f;
-            } else {
-                const int m = e / NG_K, kk = e - m * NG_K;              // consecutive threads: consecutive j (contiguous in W and Z)
-                const int j = r0 + kk;
-                const int i = m0 + m;
-                As[kk][m] = (i < wrows && j < wcols) ? abs_bf16(Wt[(size_t)i * g.cols + j]) : 0.f;
-                const int l = n0 + m;
-                Bs[kk][m] = (l < k && j < g.tn) ? Ft[(size_t)l * g.tn + j] : 0.f;
+    const uint16_t *Wt = W + (size_t)tr * g.tm * g.cols + (size_t)tc * g.tn;
+    const float *Pt = P + (size_t)tile * g.tm * k;
+    float acc[NP_KC];
+#pragma unroll
+    for (int c = 0; c < NP_KC; ++c) acc[c] = 0.f;
+    for (int i0 = 0; i0 < wrows; i0 += NP_SLAB0) {      // rows outside the matrix hold |W| = 0: nothing to add
+        uint16_t wv[RQ];
+#pragma unroll
+        for (int r = 0; r < RQ; ++r) wv[r] = (i0 + q * RQ + r < wrows && j < wcols) ? Wt[(size_t)(i0 + q * RQ + r) * g.cols + j] : (uint16_t)0;
+#pragma unroll
+        for (int u = 0; u < NP_SLAB0 * NP_KC / (NP_THREADS * NP_GROUPS); ++u) {
+            const int e = tid + NP_THREADS * NP_GROUPS * u, r = e / NP_KC, c = e - r * NP_KC;
+            Ps[r][c] = (i0 + r < g.tm && c < kc) ? Pt[(size_t)(i0 + r) * k + l0 + c] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int rr = 0; rr < RQ; ++rr) {
+            const int r = q * RQ + rr;
+            const float w = abs_bf16(wv[rr]);
+#pragma unroll
+            for (int c4 = 0; c4 < NP_KC / 4; ++c4) {
+                const float4 p = *reinterpret_cast<const float4 *>(&Ps[r][c4 * 4]);
+                acc[c4 * 4 + 0] = fmaf(p.x, w, acc[c4 * 4 + 0]);
+                acc[c4 * 4 + 1] = fmaf(p.y, w, acc[c4 * 4 + 1]);
+                acc[c4 * 4 + 2] = fmaf(p.z, w, acc[c4 * 4 + 2]);
+                acc[c4 * 4 + 3] = fmaf(p.w, w, acc[c4 * 4 + 3]);
             }
         }
         __syncthreads();
+    }
+    nmf_fold_groups(acc, red, t, q);
+    if (q == 0 && j < g.tn) {
+        float *Nt = N1 + (size_t)tile * k * g.tn;
 #pragma unroll
-        for (int kk = 0; kk < NG_K; ++kk) {
-            float a[4], b[4];
+        for (int c = 0; c < NP_KC; ++c)
+            if (c < kc) Nt[(size_t)(l0 + c) * g.tn + j] = acc[c];
+    }
+}
+
+// N2[i][l] = sum_j |W[i][j]| Z[l][j]   (tm x k per tile; the reduction runs over the tile's columns).
+// grid = (ceil(tm / 128), layer tiles, ceil(k / 32)).  A thread owns row i and 32 values of l.  A slab of 128 rows x 64
+// columns of W goes through shared memory (read along the rows, used along the columns), the slab of Z is stored
+// [column][l] so that a thread reads the 32 values of one column as eight 16-byte broadcasts.
+__global__ void __launch_bounds__(NP_THREADS * NP_GROUPS, 2)
+nmf_prod_p_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__ Z, float *__restrict__ N2)
+{
+    constexpr int WP = NP_SLAB1 + 2;                     // 33 words per row: a column is read without bank conflicts
+    constexpr int ZP = NP_KC + 4;                        // keeps rows 16-byte aligned
+    __shared__ uint16_t Ws[NP_THREADS * WP];
+    __shared__ __align__(16) float Zs[NP_SLAB1 * ZP];
+    __shared__ float red[NP_KC * NP_THREADS];
+    const int tile = blockIdx.y, tr = tile / g.gc, tc = tile - tr * g.gc, k = g.k, t = threadIdx.x, q = threadIdx.y;
+    const int tid = q * NP_THREADS + t;
+    constexpr int JQ = NP_SLAB1 / NP_GROUPS;            // columns of a slab per thread
+    const int ib = blockIdx.x * NP_THREADS, l0 = blockIdx.z * NP_KC, kc = min(NP_KC, k - l0);
+    const int wrows = min(g.tm, g.rows - tr * g.tm), wcols = min(g.tn, g.cols - tc * g.tn);
+    const uint16_t *Wt = W + (size_t)tr * g.tm * g.cols + (size_t)tc * g.tn;
+    const float *Zt = Z + (size_t)tile * k * g.tn;
+    float acc[NP_KC];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { a[u] = As[kk][ty * 4 + u]; b[u] = Bs[kk][tx * 4 + u]; }
+    for (int c = 0; c < NP_KC; ++c) acc[c] = 0.f;
+    for (int j0 = 0; j0 < wcols; j0 += NP_SLAB1) {      // columns outside the matrix hold |W| = 0
+        // (all requests of a thread go out before the first value is used: the slab costs one trip to memory, not sixteen)
+        constexpr int NW = NP_THREADS * NP_SLAB1 / (NP_THREADS * NP_GROUPS), NZ = NP_KC * NP_SLAB1 / (NP_THREADS * NP_GROUPS);
+        uint16_t wl[NW];
+        float zl[NZ];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < NW; ++u) {
+            const int e = tid + NP_THREADS * NP_GROUPS * u, r = e / NP_SLAB1, jj = e - r * NP_SLAB1;
+            wl[u] = (ib + r < wrows && j0 + jj < wcols) ? Wt[(size_t)(ib + r) * g.cols + j0 + jj] : (uint16_t)0;
+        }
 #pragma unroll
-                for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], b[v], acc[u][v]);
+        for (int u = 0; u < NZ; ++u) {
+            const int e = tid + NP_THREADS * NP_GROUPS * u, c = e / NP_SLAB1, jj = e - c * NP_SLAB1;
+            zl[u] = (c < kc && j0 + jj < g.tn) ? Zt[(size_t)(l0 + c) * g.tn + j0 + jj] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < NW; ++u) {
+            const int e = tid + NP_THREADS * NP_GROUPS * u, r = e / NP_SLAB1, jj = e - r * NP_SLAB1;
+            Ws[r * WP + jj] = wl[u];
+        }
+#pragma unroll
+        for (int u = 0; u < NZ; ++u) {
+            const int e = tid + NP_THREADS * NP_GROUPS * u, c = e / NP_SLAB1, jj = e - c * NP_SLAB1;
+            Zs[jj * ZP + c] = zl[u];
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int jj = q * JQ; jj < (q + 1) * JQ; ++jj) {
+            const float w = abs_bf16(Ws[t * WP + jj]);
+#pragma unroll
+            for (int c4 = 0; c4 < NP_KC / 4; ++c4) {
+                const float4 z = *reinterpret_cast<const float4 *>(&Zs[jj * ZP + c4 * 4]);
+                acc[c4 * 4 + 0] = fmaf(w, z.x, acc[c4 * 4 + 0]);
+                acc[c4 * 4 + 1] = fmaf(w, z.y, acc[c4 * 4 + 1]);
+                acc[c4 * 4 + 2] = fmaf(w, z.z, acc[c4 * 4 + 2]);
+                acc[c4 * 4 + 3] = fmaf(w, z.w, acc[c4 * 4 + 3]);
+            }
         }
         __syncthreads();
     }
+    nmf_fold_groups(acc, red, t, q);
+    const int i = ib + t;
+    if (q == 0 && i < g.tm) {
+        float *Nt = N2 + ((size_t)tile * g.tm + i) * k + l0;
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            const int m = m0 + ty * 4 + u, n = n0 + tx * 4 + v;
-            if (m < CM && n < CN) Ct[(size_t)m * CN + n] = acc[u][v];
-        }
+        for (int c = 0; c < NP_KC; ++c)
+            if (c < kc) Nt[c] = acc[c];
+    }
 }
 
 // G[a][b] = sum_r F(r, a) F(r, b): ZMODE 0: F = Mp [tm][k] (r = row), ZMODE 1: F = Mz [k][tn] (r = column).
-// grid = (k*k / 256, layer tiles, slices of the reduction): a block sums its slice of r and adds it to G (zeroed
-// before the launch) with one atomic per entry; a lone thread per entry over the whole reduction was measured at
-// 200-280 us per launch on the AlexNet layer, as much as the large products.
-constexpr int NMF_GRAM_SLICE = 32;
+// grid = (blocks of 32 x 32 entries, layer tiles, slices of 64 values of r): a block stages its slice of the two
+// 32-wide strips of F in shared memory, a thread sums four entries and adds them to G (zeroed before the launch)
+// with one atomic each.
+constexpr int NMF_GRAM_SLICE = 64;
 template <int ZMODE>
 __global__ void __launch_bounds__(256)
 nmf_gram_kernel(Geo g, const float *__restrict__ F, float *__restrict__ G)
 {
-    const int tile = blockIdx.y, k = g.k;
-    const int e = blockIdx.x * 256 + threadIdx.x;
-    if (e >= k * k) return;
-    const int a = e / k, b = e - a * k;
-    const float *Ft = F + (size_t)tile * (ZMODE == 0 ? (size_t)g.tm * k : (size_t)k * g.tn);
+    constexpr int GP = 33;                               // words per staged row
+    __shared__ float As[NMF_GRAM_SLICE * GP], Bs[NMF_GRAM_SLICE * GP];
+    const int tile = blockIdx.y, k = g.k, t = threadIdx.x;
+    const int kb = (k + 31) / 32;
+    const int a0 = (blockIdx.x / kb) * 32, b0 = (blockIdx.x % kb) * 32;
     const int R = ZMODE == 0 ? g.tm : g.tn;
-    const int r0 = blockIdx.z * NMF_GRAM_SLICE, r1 = min(R, r0 + NMF_GRAM_SLICE);
-    float s = 0.f;
-    for (int r = r0; r < r1; ++r)
-        s = ZMODE == 0 ? fmaf(Ft[(size_t)r * k + a], Ft[(size_t)r * k + b], s) : fmaf(Ft[(size_t)a * g.tn + r], Ft[(size_t)b * g.tn + r], s);
-    atomicAdd(G + (size_t)tile * k * k + e, s);
+    const int r0 = blockIdx.z * NMF_GRAM_SLICE;
+    const float *Ft = F + (size_t)tile * (ZMODE == 0 ? (size_t)g.tm * k : (size_t)k * g.tn);
+    for (int e = t; e < NMF_GRAM_SLICE * 32; e += 256) {
+        int r, c;
+        if (ZMODE == 0) { r = e >> 5; c = e & 31; }      // consecutive threads: consecutive rank values (contiguous in Mp)
+        else { c = e / NMF_GRAM_SLICE; r = e - c * NMF_GRAM_SLICE; }   // consecutive columns (contiguous in Mz)
+        const bool rin = r0 + r < R;
+        As[r * GP + c] = (rin && a0 + c < k) ? (ZMODE == 0 ? Ft[(size_t)(r0 + r) * k + a0 + c] : Ft[(size_t)(a0 + c) * g.tn + r0 + r]) : 0.f;
+        Bs[r * GP + c] = (rin && b0 + c < k) ? (ZMODE == 0 ? Ft[(size_t)(r0 + r) * k + b0 + c] : Ft[(size_t)(b0 + c) * g.tn + r0 + r]) : 0.f;
+    }
+    __syncthreads();
+    const int a = t >> 3, b4 = (t & 7) * 4;
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+    for (int r = 0; r < NMF_GRAM_SLICE; ++r) {
+        const float av = As[r * GP + a];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) s[u] = fmaf(av, Bs[r * GP + b4 + u], s[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        if (a0 + a < k && b0 + b4 + u < k) atomicAdd(G + (size_t)tile * k * k + (size_t)(a0 + a) * k + b0 + b4 + u, s[u]);
 }
 
 constexpr int NMF_MAX_RANK = 256;
 
-// Mz[l][j] *= N1[l][j] / (sum_m G1[l][m] Mz[m][j] + eps): a thread owns column j (the old column is read before any write).
-__global__ void __launch_bounds__(128)
+// Mz[l][j] *= N1[l][j] / (sum_m G1[l][m] Mz[m][j] + eps).  A block holds the old values of its columns of Mz in shared
+// memory ([k][columns]); a thread owns column j and forms four denominators at a time, reading row m of the
+// (symmetric) Gram matrix as G1[m][l .. l+3].
+__global__ void
 nmf_update_z_kernel(Geo g, const float *__restrict__ N1, const float *__restrict__ G1, float *__restrict__ Z, float eps)
 {
-    const int tile = blockIdx.y, k = g.k, j = blockIdx.x * 128 + threadIdx.x;
-    if (j >= g.tn) return;
+    extern __shared__ __align__(16) float nmf_old[];    // [k][blockDim.x]
+    const int tile = blockIdx.y, k = g.k, t = threadIdx.x, nb = blockDim.x, j = blockIdx.x * nb + t;
     float *Zt = Z + (size_t)tile * k * g.tn;
     const float *Nt = N1 + (size_t)tile * k * g.tn, *Gt = G1 + (size_t)tile * k * k;
-    float z[NMF_MAX_RANK];
-    for (int m = 0; m < k; ++m) z[m] = Zt[(size_t)m * g.tn + j];
-    for (int l = 0; l < k; ++l) {
-        float den = 0.f;
-        for (int m = 0; m < k; ++m) den = fmaf(__ldg(Gt + l * k + m), z[m], den);
-        Zt[(size_t)l * g.tn + j] = z[l] * Nt[(size_t)l * g.tn + j] / (den + eps);
+    for (int m0 = 0; m0 < k; m0 += 8) {                  // eight requests in flight per thread
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = (m0 + u < k && j < g.tn) ? Zt[(size_t)(m0 + u) * g.tn + j] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (m0 + u < k) nmf_old[(m0 + u) * nb + t] = v[u];
+    }
+    __syncthreads();
+    if (j >= g.tn) return;
+    const bool vec = (k & 3) == 0;
+    for (int l0 = 0; l0 < k; l0 += 4) {
+        float nv[4];                                     // the numerators are asked for before the sums they divide
+#pragma unroll
+        for (int u = 0; u < 4; ++u) nv[u] = l0 + u < k ? Nt[(size_t)(l0 + u) * g.tn + j] : 0.f;
+        float den[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+        for (int m = 0; m < k; ++m) {
+            const float z = nmf_old[m * nb + t];
+            if (vec) {
+                const float4 gv = __ldg(reinterpret_cast<const float4 *>(Gt + (size_t)m * k + l0));
+                den[0] = fmaf(gv.x, z, den[0]); den[1] = fmaf(gv.y, z, den[1]);
+                den[2] = fmaf(gv.z, z, den[2]); den[3] = fmaf(gv.w, z, den[3]);
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (l0 + u < k) den[u] = fmaf(__ldg(Gt + (size_t)(l0 + u) * k + m), z, den[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (l0 + u < k) Zt[(size_t)(l0 + u) * g.tn + j] = nmf_old[(l0 + u) * nb + t] * nv[u] / (den[u] + eps);
     }
 }
 
-// Mp[i][l] *= N2[i][l] / (sum_m Mp[i][m] G2[m][l] + eps): a thread owns row i.
-__global__ void __launch_bounds__(128)
+// Mp[i][l] *= N2[i][l] / (sum_m Mp[i][m] G2[m][l] + eps).  The block's rows of Mp (contiguous in memory) are staged in
+// shared memory, k + 1 words apart; a thread owns row i.
+__global__ void
 nmf_update_p_kernel(Geo g, const float *__restrict__ N2, const float *__restrict__ G2, float *__restrict__ P, float eps)
 {
-    const int tile = blockIdx.y, k = g.k, i = blockIdx.x * 128 + threadIdx.x;
+    extern __shared__ __align__(16) float nmf_old[];    // [blockDim.x][k + 1]
+    const int tile = blockIdx.y, k = g.k, t = threadIdx.x, nb = blockDim.x, ib = blockIdx.x * nb, i = ib + t;
+    float *Pt = P + (size_t)tile * g.tm * k;
+    const float *Nt = N2 + (size_t)tile * g.tm * k, *Gt = G2 + (size_t)tile * k * k;
+    const int nrows = min(nb, g.tm - ib);
+    for (int e = t; e < nrows * k; e += nb) {
+        const int r = e / k, c = e - r * k;
+        nmf_old[r * (k + 1) + c] = Pt[(size_t)ib * k + e];
+    }
+    __syncthreads();
     if (i >= g.tm) return;
-    float *Pt = P + ((size_t)tile * g.tm + i) * k;
-    const float *Nt = N2 + ((size_t)tile * g.tm + i) * k, *Gt = G2 + (size_t)tile * k * k;
-    float p[NMF_MAX_RANK];
-    for (int m = 0; m < k; ++m) p[m] = Pt[m];
-    for (int l = 0; l < k; ++l) {
-        float den = 0.f;
-        for (int m = 0; m < k; ++m) den = fmaf(p[m], __ldg(Gt + m * k + l), den);
-        Pt[l] = p[l] * Nt[l] / (den + eps);
+    const float *mine = nmf_old + t * (k + 1);
+    const bool vec = (k & 3) == 0;
+    for (int l0 = 0; l0 < k; l0 += 4) {
+        float nv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) nv[u] = l0 + u < k ? Nt[(size_t)i * k + l0 + u] : 0.f;
+        float den[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+        for (int m = 0; m < k; ++m) {
+            const float p = mine[m];
+            if (vec) {
+                const float4 gv = __ldg(reinterpret_cast<const float4 *>(Gt + (size_t)m * k + l0));
+                den[0] = fmaf(p, gv.x, den[0]); den[1] = fmaf(p, gv.y, den[1]);
+                den[2] = fmaf(p, gv.z, den[2]); den[3] = fmaf(p, gv.w, den[3]);
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (l0 + u < k) den[u] = fmaf(p, __ldg(Gt + (size_t)m * k + l0 + u), den[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (l0 + u < k) Pt[(size_t)i * k + l0 + u] = mine[l0 + u] * nv[u] / (den[u] + eps);
     }
 }
 
@@ -143,16 +302,19 @@ lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, in
     const long long tiles = (long long)g.gr * g.gc;
     if (tiles > 65535) return LRBI_ERR_UNSUPPORTED;
     float *N = ws, *G = ws + (size_t)tiles * g.k * (g.tm > g.tn ? g.tm : g.tn);
-    const unsigned kt = (unsigned)((g.k + NG_T - 1) / NG_T), gk2 = (unsigned)((g.k * g.k + 255) / 256);
+    const unsigned kc = (unsigned)((g.k + NP_KC - 1) / NP_KC), kb = (unsigned)((g.k + 31) / 32);
+    // the update kernels keep k x (threads) old values in shared memory: 128 threads up to rank 64, 32 above
+    const unsigned ut = g.k <= 64 ? 128u : 32u;
+    const size_t smem_z = (size_t)g.k * ut * sizeof(float), smem_p = (size_t)ut * (g.k + 1) * sizeof(float);
     for (int it = 0; it < iterations; ++it) {
-        nmf_gemm_kernel<0><<<dim3((unsigned)((g.tn + NG_T - 1) / NG_T), kt, (unsigned)tiles), 256, 0, s>>>(g, W, mp, N);
+        nmf_prod_z_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mp, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
-        nmf_gram_kernel<0><<<dim3(gk2, (unsigned)tiles, (unsigned)((g.tm + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mp, G);
-        nmf_update_z_kernel<<<dim3((unsigned)((g.tn + 127) / 128), (unsigned)tiles), 128, 0, s>>>(g, N, G, mz, eps);
-        nmf_gemm_kernel<1><<<dim3(kt, (unsigned)((g.tm + NG_T - 1) / NG_T), (unsigned)tiles), 256, 0, s>>>(g, W, mz, N);
+        nmf_gram_kernel<0><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tm + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mp, G);
+        nmf_update_z_kernel<<<dim3((unsigned)((g.tn + ut - 1) / ut), (unsigned)tiles), ut, smem_z, s>>>(g, N, G, mz, eps);
+        nmf_prod_p_kernel<<<dim3((unsigned)((g.tm + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mz, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
-        nmf_gram_kernel<1><<<dim3(gk2, (unsigned)tiles, (unsigned)((g.tn + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mz, G);
-        nmf_update_p_kernel<<<dim3((unsigned)((g.tm + 127) / 128), (unsigned)tiles), 128, 0, s>>>(g, N, G, mp, eps);
+        nmf_gram_kernel<1><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tn + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mz, G);
+        nmf_update_p_kernel<<<dim3((unsigned)((g.tm + ut - 1) / ut), (unsigned)tiles), ut, smem_p, s>>>(g, N, G, mp, eps);
         count_launch(6);
     }
     const cudaError_t e = cudaGetLastError();
