@@ -670,6 +670,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             ok = mbar_wait(&ctl->bits_ready[0], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
             if (ok) ok = mbar_wait(&ctl->bits_ready[1], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
         }
+        // The lanes of a warp leave a barrier wait one by one (each polls for itself); the tensor-memory loads of the
+        // epilogue are warp-wide instructions and need the warp back together, with one verdict for all its lanes.
+        ok = __all_sync(0xFFFFFFFFu, ok);
         if (ok && PERSIST) {
             // The operand stages already belong to the next tile: every warp moves its 32 output features x 16
             // (fp32: 8) batch columns through 1 KB of its own and stores 16-byte pieces, 64 (128) bytes of a row of Y
