@@ -386,6 +386,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     __syncthreads();
     // Both CTAs' barriers must exist before anyone signals across.  Everybody arrives at the cluster barrier now; the
     // warp of the TMA producer waits only after its first round of copies is on its way (they touch this CTA alone).
+    __syncwarp();                                        // (the cluster barrier is a warp-wide instruction)
     if (PAIR) {
         cluster_arrive();
         if (warp != 0) cluster_wait();
@@ -788,6 +789,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
+    __syncwarp();                    // (warp-wide instructions follow; a warp's lanes may have come here on different paths)
     if (PAIR) cluster_sync_all();    // neither CTA frees tensor memory or leaves while the other may still touch it
     if (warp == 1) {
         tc_fence_after();
