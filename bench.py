@@ -467,6 +467,8 @@ def run_ours(args):
             if name == args.workload and (ob == batch or not ob):
                 continue                                  # the headline workload itself
             ow = setup_workload(B, name, ob)
+            if os.environ.get("LRBI_BENCH_TRACE"):
+                print("timing %s %s" % (name, ob), file=sys.stderr, flush=True)
             l0 = B.launch_count()
             ts = time_calls(ow["step"], args.other_steps, 3, flush2)
             nl = (B.launch_count() - l0) / (args.other_steps + 3)

@@ -329,15 +329,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u; // 0 = leader of the pair
     // grid.x runs fastest over blocks that share rows of W, so W streams from HBM once and X stays in L2.
     // Pair mode: the two CTAs of a cluster are neighbours along x (x = 2 * batch tile + rank), y = 256-row pair.
-    // PERSIST: the block's n-th tile is tile t = (pair index) + n * (pairs in the grid); t runs fastest over batch tiles.
+    // PERSIST: the block's n-th tile is tile t = (pair index) + n * (pairs in the grid).  t runs fastest over the tiles of
+    // the smaller operand (batch tiles when X is the smaller matrix, row pairs when W is), so that the pairs at work
+    // at any time share all of the small operand, which stays in L2, and the large one streams from memory once.
     const int nbt = (batch + BN - 1) / BN;
+    const int nrp = (g.rows + 2 * TC_BM - 1) / (2 * TC_BM);
+    const bool rows_fast = g.rows < batch;
     const int tile_first = PERSIST ? (int)(blockIdx.x >> 1) : 0, tile_step = PERSIST ? (int)(gridDim.x >> 1) : 1;
-    const int my_tiles = PERSIST ? (nbt * ((g.rows + 2 * TC_BM - 1) / (2 * TC_BM)) - tile_first + tile_step - 1) / tile_step : 1;
+    const int my_tiles = PERSIST ? (nbt * nrp - tile_first + tile_step - 1) / tile_step : 1;
     auto tile_b0 = [&](int n) {                          // first batch row of the block's n-th tile
-        return PERSIST ? ((tile_first + n * tile_step) % nbt) * BN : (int)(PAIR ? (blockIdx.x >> 1) : blockIdx.x) * BN;
+        const int t = tile_first + n * tile_step;
+        return PERSIST ? (rows_fast ? t / nrp : t % nbt) * BN : (int)(PAIR ? (blockIdx.x >> 1) : blockIdx.x) * BN;
     };
     auto tile_o0 = [&](int n) {                          // first row of W of this block in its n-th tile
-        return PERSIST ? (((tile_first + n * tile_step) / nbt) * 2 + (int)rank) * TC_BM
+        const int t = tile_first + n * tile_step;
+        return PERSIST ? ((rows_fast ? t % nrp : t / nbt) * 2 + (int)rank) * TC_BM
                        : (int)(PAIR ? (blockIdx.y * 2 + rank) : blockIdx.y) * TC_BM;
     };
     const int b0 = tile_b0(0), o0 = tile_o0(0);
@@ -597,9 +603,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         // ------------------------------------------------------------- pruning warps
         const int mt = threadIdx.x - 64;                // 0..255
         const int mw = mt >> 5;                         // pruning warp 0..7
-        // The warps form two sets of four that take alternate K blocks (set q: the blocks whose running number is
-        // q mod 2), so the wait - load - prune - store - fence - arrive chain of one K block overlaps the next
-        // block's: the chain is latency, not work, and one set alone was measured at half a microsecond per block.
+        // The warps form two sets of four; set q takes the K blocks that land in the stages with s mod 2 == q, so the
+        // wait - load - prune - store - fence - arrive chain of one K block overlaps the next block's (the chain is
+        // latency, not work).  The split goes by stage, not by K block, on purpose: a stage's barriers are then waited
+        // on by the same warps in every phase.  A warp that skipped a phase of a barrier would ask for a parity that
+        // the barrier's previous phase also has, and pass before the copies it waits for were even issued (with an
+        // odd number of stages and sets by K block that happened about once in two hundred launches).
         // Inside a set a thread owns one row of the 128 (eight 16-byte chunks; the eight lanes of one access phase
         // fall on eight different swizzled chunk positions).
         const int set = mw >> 2;
@@ -611,7 +620,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         int kp = 0;                                      // K block inside its panel
         int P = 0;                                       // panel index, counted across the block's tiles
         int P_seen = -1;                                 // last panel whose index bits this warp has waited for
-        uint32_t G = 0;                                  // running number of the K block, across the block's tiles
         auto panel_bits_ready = [&]() {                  // (every warp waits for every panel, also one it takes no block of:
             if (P_seen != P) {                           //  its arrival below must not run ahead of the decoders)
                 ok = mbar_wait(&ctl->bits_ready[P & 1], (P >> 1) & 1, abort_flag, status, DEV_TIMEOUT_FULL);
@@ -620,8 +628,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
         };
         for (int tile_n = 0; tile_n < my_tiles && ok; ++tile_n) {
         const int b0 = tile_b0(tile_n), o0 = tile_o0(tile_n);
-        for (int it = 0; it < nkb && ok; ++it, ++G) {
-            const bool mine = (G & 1u) == (uint32_t)set;
+        for (int it = 0; it < nkb && ok; ++it) {
+            const bool mine = (s & 1) == set;
             if (DW) {                                    // nothing is pruned inside this contraction: pass the stage on
                 if (mine) {
                     ok = mbar_wait(&ctl->full[s], full_parity, abort_flag, status, DEV_TIMEOUT_FULL);
@@ -747,8 +755,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             if (DW) P += 2;
         }
         if (ok && !PERSIST) {
-            // K split: the kernel that adds the partial sums up may be set up from here on (it waits for this grid's end)
-            if (partials != nullptr && mt == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             tc_fence_after();
             // All MMAs have completed.  In tensor memory a lane is an output feature and a column a batch row, so the 32
             // lanes of a warp hold 32 consecutive outputs of one row of Y: every column goes out as one 64-byte (fp32:
@@ -830,9 +836,6 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ partials, int splits, long long n, void *__restrict__ Y, int y_dtype)
 {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    // launched while the product kernel is still draining (programmatic dependent launch): its writes are
-    // visible only after this wait
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (idx >= n) return;
     float acc = 0.f;
     for (int z = 0; z < splits; ++z) acc += partials[(long long)z * n + idx];
@@ -1043,20 +1046,9 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
     if (plan.splits > 1) {
         const long long n = (long long)batch * g.rows;
-        // the reduction's blocks may be set up while the product kernel's last blocks finish; they wait for its
-        // completion before they read (griddepcontrol.wait)
-        cudaLaunchConfig_t rcfg = {};
-        rcfg.gridDim = dim3((unsigned)((n + 255) / 256));
-        rcfg.blockDim = dim3(256);
-        rcfg.stream = s;
-        cudaLaunchAttribute rattr[1];
-        rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        rattr[0].val.programmaticStreamSerializationAllowed = 1;
-        rcfg.attrs = rattr;
-        rcfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&rcfg, splitk_reduce_kernel, (const float *)partials, (int)plan.splits, n, Y, y_dtype);
+        splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, plan.splits, n, Y, y_dtype);
         count_launch();
-        if (e == cudaSuccess) e = cudaGetLastError();
+        e = cudaGetLastError();
         if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
     }
     return LRBI_OK;
