@@ -758,6 +758,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
             if (DW) P += 2;
         }
         if (epi_ok && !PERSIST) {
+            // K split: the kernel that adds the partial sums up may be set up from here on (it waits for this grid's end)
+            if (partials != nullptr && mt == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             tc_fence_after();
             // All MMAs have completed.  In tensor memory a lane is an output feature and a column a batch row, so the 32
             // lanes of a warp hold 32 consecutive outputs of one row of Y: every column goes out as one 64-byte (fp32:
@@ -839,6 +841,9 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ partials, int splits, long long n, void *__restrict__ Y, int y_dtype)
 {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    // launched while the product kernel is still draining (programmatic dependent launch): its writes are
+    // visible only after this wait
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (idx >= n) return;
     float acc = 0.f;
     for (int z = 0; z < splits; ++z) acc += partials[(long long)z * n + idx];
@@ -1049,9 +1054,20 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
     if (plan.splits > 1) {
         const long long n = (long long)batch * g.rows;
-        splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, plan.splits, n, Y, y_dtype);
+        // the reduction's blocks may be set up while the product kernel's last blocks finish; they wait for its
+        // completion before they read (griddepcontrol.wait)
+        cudaLaunchConfig_t rcfg = {};
+        rcfg.gridDim = dim3((unsigned)((n + 255) / 256));
+        rcfg.blockDim = dim3(256);
+        rcfg.stream = s;
+        cudaLaunchAttribute rattr[1];
+        rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        rattr[0].val.programmaticStreamSerializationAllowed = 1;
+        rcfg.attrs = rattr;
+        rcfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&rcfg, splitk_reduce_kernel, (const float *)partials, (int)plan.splits, n, Y, y_dtype);
         count_launch();
-        e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }
     }
     return LRBI_OK;
