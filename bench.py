@@ -31,16 +31,18 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, one launch, from the ncu capture
 # summarised under profiles/ (null for workloads without a capture of the current kernel)
 NCU_TRAFFIC_BYTES = {
-    ("ffn_16384x4096", 4096): 401_400_000,      # 285.8 MB read + 115.6 MB written (profiles/gemm_tc_pair2_ffn_16384x4096.md)
-    ("lenet_fc1", 32): 1_050_000,
-    ("decode_4096", 0): 534_000,                # the 2 MiB mask is still in L2 when the kernel ends
-    ("decode_32768", 0): 104_200_000,
+    ("ffn_16384x4096", 4096): 403_700_000,      # 292.0 MB read + 111.7 MB written (profiles/gemm_tc_pair2_ffn_16384x4096.md)
+    ("lenet_fc1", 32): 1_050_000,               # both launches (K-split kernel + reduction)
+    ("decode_4096", 0): 530_000,                # the 2 MiB mask is still in L2 when the kernel ends
+    ("decode_32768", 0): 104_000_000,
     ("alexnet_fc", 1): 76_200_000,
-    ("alexnet_fc", 16): 78_900_000,             # both launches (K-split kernel + reduction)
-    ("alexnet_fc", 128): 97_500_000,
+    ("alexnet_fc", 16): 78_900_000,             # both launches
+    ("alexnet_fc", 128): 97_800_000,            # both launches
     ("conv3x3_256", 12544): 59_100_000,         # Y (6.4 MB) is still in L2 when the kernel ends
     ("alexnet_fc", -1): 76_200_000,
-    ("ffn_16384x4096", -1): 135_500_000,
+    ("ffn_16384x4096", -1): 135_800_000,
+    ("ffn_16384x4096", -2): 432_300_000,        # dX: 412.4 MB read + 19.9 MB written
+    ("ffn_16384x4096", -3): 432_700_000,        # dW: the product kernel alone, 316.5 MB read + 116.2 MB written
 }
 # The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
 # batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
