@@ -42,7 +42,6 @@ NCU_TRAFFIC_BYTES = {
     ("alexnet_fc", -1): 76_200_000,
     ("ffn_16384x4096", -1): 135_800_000,
     ("ffn_16384x4096", -2): 432_300_000,        # dX: 412.4 MB read + 19.9 MB written
-    ("ffn_16384x4096", -3): 432_700_000,        # dW: the product kernel alone, 316.5 MB read + 116.2 MB written
 }
 # The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
 # batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
@@ -232,7 +231,7 @@ def kernel_label(B, layer, batch):
         return "decode"
     if batch < 0:
         return {-1: "index_cost", -2: "backward dX (forward kernel on the transposed layer)",
-                -3: "backward dW (2 transposes + persistent pair kernel, index applied in the epilogue)",
+                -3: "backward dW (persistent pair kernel on MN-major dY and X, index applied in the epilogue)",
                 -4: "nmf, one multiplicative update of Mz and Mp (fp32 CUDA cores)"}[batch]
     plan = B.masked_gemm_plan(layer, batch)
     name = B.ALGO_NAMES[plan.algo]

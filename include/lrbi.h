@@ -290,11 +290,14 @@ LRBI_API lrbi_status lrbi_nmf_update(const lrbi_layout *layout, const uint16_t *
  *       kernels: the packed factors are used as they are (a row word of Ip is a column word of Ip^T).  algo:
  *       LRBI_ALGO_AUTO, _GENERIC or _TENSOR / _TENSOR_PAIR / _TENSOR_PAIR2 / _TENSOR_PAIR192 (tensor-core shapes: rows % 8 == 0, and
  *       tile_cols % 128 == 0 and tile_rows % 64 == 0 unless the grid has one tile in that direction).
- * lrbi_masked_gemm_dw   dY [batch][rows], X [batch][cols] -> dW [rows][cols].  `workspace` is DEVICE memory of at least
- *       lrbi_masked_gemm_dw_workspace(layout, batch) bytes, 16-byte aligned, owned by the caller, scratch for the
- *       call (transposed copies of dY and X): the contraction runs on the tensor-core kernel with nothing pruned
- *       inside it, and the index, decoded on the fly and never stored, is applied as dW is written (large aligned
- *       shapes) or to dW in place afterwards.  batch % 8 != 0 or a NULL workspace falls back to a slow
+ * lrbi_masked_gemm_dw   dY [batch][rows], X [batch][cols] -> dW [rows][cols].  Large aligned layers (rows, cols and
+ *       batch multiples of 8; tile_cols % 128 == 0 and tile_rows % 256 == 0 unless the grid has one tile in that
+ *       direction) run as ONE launch of the tensor-core kernel on dY and X as they are (the operands are read
+ *       MN-major): nothing is pruned inside the contraction and the index, decoded on the fly and never stored, is
+ *       applied as dW is written; `workspace` is not touched and may be NULL.  Other tensor-core shapes use
+ *       `workspace` (DEVICE memory of at least lrbi_masked_gemm_dw_workspace(layout, batch) bytes, 16-byte aligned,
+ *       owned by the caller, scratch for the call) for transposed copies of dY and X and apply the index to dW in
+ *       place afterwards; batch % 8 != 0, or a NULL workspace on such a shape, falls back to a slow
  *       one-thread-per-weight kernel.
  * lrbi_transpose_bf16   dst [cols][rows] = transpose of src [rows][cols] (bf16 bit patterns; dst must not overlap src).
  */

@@ -309,6 +309,12 @@ lrbi_status lrbi_masked_gemm_dw(const lrbi_layout *layout, const uint16_t *dY, c
     // the contraction as a forward product: "weights" X^T [cols][batch], "activations" dY^T [rows][batch], one tile of rank one
     lrbi_layout one = {layout->cols, batch, layout->cols, batch, 1};
     const Geo g1 = make_geo(one);
+    // First choice: the persistent pair kernel on X and dY as they are (MN-major operands), nothing pruned inside the
+    // contraction, the index (seen transposed: rows = layer columns) applied as the output tile is stored.
+    if ((batch % 8) == 0 && gemm_tc_supported(g1, layout->rows)) {
+        const lrbi_status st0 = launch_gemm_tc_dw(g1, transposed_geo(g), X, iz, ip, dY, layout->rows, dW, dw_dtype, s, true);
+        if (st0 != LRBI_ERR_UNSUPPORTED) return st0;
+    }
     if (!workspace || (batch % 8) != 0 || !gemm_tc_supported(g1, layout->rows))
         return launch_dw_generic(g, dY, X, batch, ip, iz, dW, dw_dtype, s);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
@@ -319,8 +325,7 @@ lrbi_status lrbi_masked_gemm_dw(const lrbi_layout *layout, const uint16_t *dY, c
     lrbi_status st = launch_transpose_bf16(dY, batch, layout->rows, dYt, s);
     if (st == LRBI_OK) st = launch_transpose_bf16(X, batch, layout->cols, Xt, s);
     if (st != LRBI_OK) return st;
-    // First choice: the persistent pair kernel with nothing pruned inside the contraction and the index (seen transposed:
-    // rows = layer columns) applied as the output tile is stored.
+    // (kept for layers whose row count is not a multiple of 8) the same kernel on transposed copies
     st = launch_gemm_tc_dw(g1, transposed_geo(g), Xt, iz, ip, dYt, layout->rows, dW, dw_dtype, s);
     if (st != LRBI_ERR_UNSUPPORTED) return st;
     // Otherwise: the forward kernel with an all-ones index of rank one, then the index applied to dW in place.

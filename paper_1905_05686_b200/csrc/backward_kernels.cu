@@ -6,10 +6,11 @@
 //        (the row words of Ip are the column words of Ip^T and the other way round, so the packed arrays are used as
 //        they are, with the tile grid walked column-major);
 //   dW   is the product with X^T in the place of the weights and dY^T as the activations, on the persistent pair
-//        kernel in its DW mode: nothing is pruned inside the contraction, the index of every output tile is decoded
-//        from the layer's factors (seen through the transposed layout) while the tile accumulates, and the epilogue
-//        writes zeros where Ia = 0.  Shapes that kernel does not take run the same product with an index of rank
-//        one whose bits are all set, followed by apply_index on dW in place.
+//        kernel in its DW mode: X and dY are read as they are (MN-major operands of the MMA), nothing is pruned inside
+//        the contraction, the index of every output tile is decoded from the layer's factors (seen through the
+//        transposed layout) while the tile accumulates, and the epilogue writes zeros where Ia = 0.  Layers whose row
+//        count is not a multiple of 8 run the same kernel on transposed copies; shapes that kernel does not take run
+//        the product with an index of rank one whose bits are all set, followed by apply_index on dW in place.
 // This file holds the helper kernels: the bf16 transpose, the in-place application of the index, a filler, and a
 // slow any-shape dW.
 #include "lrbi_common.cuh"

@@ -144,6 +144,19 @@ __device__ __forceinline__ uint64_t make_sw128_desc(uint32_t saddr)
     d |= (uint64_t)2 << 61;                             // 128-byte swizzle
     return d;
 }
+// The same for an MN-major operand (the M or N index runs along memory, K across rows), 128-byte swizzle: an atom is
+// 64 values of M/N (128 bytes) x 8 values of K (rows 128 bytes apart); atoms along M/N lie `mn_atom_bytes` apart
+// (the leading byte offset), groups of 8 values of K 1024 bytes apart (the stride byte offset).
+__device__ __forceinline__ uint64_t make_sw128_mn_desc(uint32_t saddr, uint32_t mn_atom_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(mn_atom_bytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = bn.
 __host__ __device__ constexpr uint32_t make_idesc(int bn, int m = TC_BM)
 {
@@ -282,7 +295,7 @@ __device__ __forceinline__ int warp_of_thread_decoder_group(unsigned tid)
 // pruned inside the contraction (the pruning warps only pass the stages on); `gi` is the layout of the index as the
 // output sees it (rows = rows of the output tile, columns = its batch axis), the decoders decode the two 256-column
 // panels of each output tile from it, and the epilogue zeroes the pruned outputs as it stores them.
-template <int BN, int PW, bool PAIR, bool PERSIST, bool DW>
+template <int BN, int PW, bool PAIR, bool PERSIST, bool DW, bool MNM>
 __global__ void __launch_bounds__(tc_threads(BN), (BN > 256 || BN == 192) ? 1 : 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map, Geo g, Geo gi, TileRanks rk,
                const uint32_t *__restrict__ ip, const uint32_t *__restrict__ iz, int batch,
@@ -304,6 +317,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     constexpr int MMA_N = PAIR ? (BN < 256 ? BN : 256) : BN;
     static_assert(!PAIR || BN == 192 || BN == 256 || BN == 512, "pair mode: one accumulator of 192 or 256 columns, or two of 256");
     static_assert(!PERSIST || BN == 512, "the persistent epilogue walks two 256-column accumulators");
+    static_assert(!MNM || (DW && PERSIST && PAIR), "MN-major operands: the weight-gradient product only");
     constexpr int KBP = PW / 2;                          // K blocks per panel
     uint8_t *a_base = smem;
     uint8_t *b_base = smem + (size_t)stages * TC_A_STAGE_BYTES;
@@ -413,11 +427,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 const int b0 = tile_b0(n), o0 = tile_o0(n);
                 if (!mbar_wait(&ctl->empty[s], parity, abort_flag, status, DEV_TIMEOUT_EMPTY)) { go = false; break; }
                 mbar_arrive_expect_tx(&ctl->full[s], B_STAGE_BYTES + TC_A_STAGE_BYTES);
+                if (MNM) {
+                    // MN-major operands: boxes of 64 values of M (or N) x 64 values of K, 8 KB each; this CTA's 128
+                    // rows of A are two boxes, its 128 columns of accumulator a two more
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d(a_base + s * TC_A_STAGE_BYTES + h * 8192, &w_map, &ctl->full[s], o0 + 64 * h, (kb_begin + it) * TC_BK);
+#pragma unroll
+                    for (int a = 0; a < NACC; ++a)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_2d(b_base + s * B_STAGE_BYTES + a * 16384 + h * 8192, &x_map, &ctl->full[s],
+                                        b0 + a * 256 + (int)rank * 128 + 64 * h, (kb_begin + it) * TC_BK);
+                } else {
                 tma_load_2d(a_base + s * TC_A_STAGE_BYTES, &w_map, &ctl->full[s], (kb_begin + it) * TC_BK, o0);
 #pragma unroll
                 for (int a = 0; a < NACC; ++a)
                     tma_load_2d(b_base + s * B_STAGE_BYTES + a * (XBOX_ROWS * TC_BK * 2), &x_map, &ctl->full[s],
                                 (kb_begin + it) * TC_BK, b0 + a * 256 + (int)rank * XBOX_ROWS);
+                }
                 issued = true;
                 if (++s == stages) { s = 0; parity ^= 1; }
             }
@@ -439,7 +467,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = PAIR ? make_idesc(MMA_N, 2 * TC_BM) : make_idesc(MMA_N);
+            constexpr uint32_t idesc = (PAIR ? make_idesc(MMA_N, 2 * TC_BM) : make_idesc(MMA_N)) | (MNM ? (1u << 15) | (1u << 16) : 0u);   // bits 15, 16: A, B MN-major
             bool ok = true;
             int s = 0;
             uint32_t parity = 0;
@@ -455,12 +483,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant_
                 ok = mbar_wait(&ctl->masked[s], parity, abort_flag, status, DEV_TIMEOUT_FULL);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t da = make_sw128_desc(smem_u32(a_base + s * TC_A_STAGE_BYTES));
-                const uint64_t db = make_sw128_desc(smem_u32(b_base + s * B_STAGE_BYTES));
+                const uint64_t da = MNM ? make_sw128_mn_desc(smem_u32(a_base + s * TC_A_STAGE_BYTES), 8192)
+                                        : make_sw128_desc(smem_u32(a_base + s * TC_A_STAGE_BYTES));
+                const uint64_t db = MNM ? make_sw128_mn_desc(smem_u32(b_base + s * B_STAGE_BYTES), 8192)
+                                        : make_sw128_desc(smem_u32(b_base + s * B_STAGE_BYTES));
 #pragma unroll
                 for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
                     // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in address units
-                    if (PAIR) {
+                    if (MNM) {                           // 16 values of K further: 16 rows of 128 bytes
+#pragma unroll
+                        for (int a = 0; a < NACC; ++a)
+                            umma2_bf16(tmem_d + (uint32_t)(a * 256), da + (uint64_t)(128 * k4),
+                                       db + (uint64_t)(a * (16384 >> 4) + 128 * k4), idesc, (it | k4) ? 1u : 0u);
+                    } else if (PAIR) {
 #pragma unroll
                         for (int a = 0; a < NACC; ++a)   // box a of the B stage -> accumulator a (256 columns further)
                             umma2_bf16(tmem_d + (uint32_t)(a * 256), da + (uint64_t)(2 * k4),
@@ -996,7 +1031,7 @@ static int device_sm_count(int *dev_out)
     return sm_count;
 }
 
-template <int BN, int PW, bool PAIR, bool PERSIST, bool DW = false>
+template <int BN, int PW, bool PAIR, bool PERSIST, bool DW = false, bool MNM = false>
 static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const uint16_t *W, const uint32_t *ip,
                              const uint32_t *iz, const uint16_t *X, int batch, void *Y, int y_dtype,
                              cudaStream_t s, float *partials, const TileRanks &rk, const Geo *index_geo = nullptr)
@@ -1005,23 +1040,25 @@ static lrbi_status launch_tc(const Geo &g, const TcPlan &plan, int dev, const ui
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) { note_cuda_error(-1); return LRBI_ERR_CUDA; }
     CUtensorMap map;
-    const cuuint64_t dims[2] = {(cuuint64_t)g.cols, (cuuint64_t)batch};
-    const cuuint64_t strides[1] = {(cuuint64_t)g.cols * 2};
-    const cuuint32_t box[2] = {TC_BK, PAIR ? (BN < 256 ? BN / 2 : 128) : BN};
+    // K-major operands: [rows of the operand][K]; MN-major (MNM): [K][rows of the operand], boxes of 64 x 64
+    const cuuint64_t dims[2] = {(cuuint64_t)(MNM ? batch : g.cols), (cuuint64_t)(MNM ? g.cols : batch)};
+    const cuuint64_t strides[1] = {(cuuint64_t)(MNM ? batch : g.cols) * 2};
+    const cuuint32_t box[2] = {TC_BK, MNM ? TC_BK : PAIR ? (BN < 256 ? BN / 2 : 128) : BN};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
     CUtensorMap wmap;
-    const cuuint64_t wdims[2] = {(cuuint64_t)g.cols, (cuuint64_t)g.rows};
-    const cuuint32_t wbox[2] = {TC_BK, TC_BM};
-    r = encode(&wmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(W), wdims, strides, wbox, estr,
+    const cuuint64_t wdims[2] = {(cuuint64_t)(MNM ? g.rows : g.cols), (cuuint64_t)(MNM ? g.cols : g.rows)};
+    const cuuint64_t wstrides[1] = {(cuuint64_t)(MNM ? g.rows : g.cols) * 2};
+    const cuuint32_t wbox[2] = {TC_BK, MNM ? TC_BK : TC_BM};
+    r = encode(&wmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(W), wdims, wstrides, wbox, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { note_cuda_error((int)r); return LRBI_ERR_CUDA; }
 
-    auto kern = gemm_tc_kernel<BN, PW, PAIR, PERSIST, DW>;
+    auto kern = gemm_tc_kernel<BN, PW, PAIR, PERSIST, DW, MNM>;
     {
         // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the function
         static bool attr_done[LRBI_MAX_DEVICES] = {false};
@@ -1118,9 +1155,12 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
 // Xt [layer cols][batch]; reduction over the batch; "batch" = rows of the layer, read from dYt [layer rows][batch]), `gi`
 // the index as the output tile sees it (the layer's layout transposed).  Returns LRBI_ERR_UNSUPPORTED when the shape
 // does not run on that kernel (the caller then takes another route).
+// mn_major: the operands are X [batch][layer cols] and dY [batch][layer rows] as the layer has them (the M and the N
+// index run along memory, K across rows); no transposed copies are needed.  Needs layer rows % 8 == 0.
 lrbi_status launch_gemm_tc_dw(const Geo &g, const Geo &gi, const uint16_t *Xt, const uint32_t *ip_t, const uint32_t *iz_t,
-                              const uint16_t *dYt, int out_rows, void *dW, int dtype, cudaStream_t s)
+                              const uint16_t *dYt, int out_rows, void *dW, int dtype, cudaStream_t s, bool mn_major)
 {
+    if (mn_major && ((out_rows % 8) != 0 || (g.rows % 8) != 0)) return LRBI_ERR_UNSUPPORTED;   // 16-byte rows for the copies
     if (!gemm_tc_supported(g, out_rows) || gi.k > TC_MAX_RANK) return LRBI_ERR_UNSUPPORTED;
     if (!(gi.gr == 1 || (gi.tm % TC_BM) == 0) || !(gi.gc == 1 || (gi.tn % 256) == 0)) return LRBI_ERR_UNSUPPORTED;
     int dev = -1;
@@ -1132,6 +1172,7 @@ lrbi_status launch_gemm_tc_dw(const Geo &g, const Geo &gi, const uint16_t *Xt, c
     if (!make_tc_plan(gs, out_rows, sm_count, 2, &plan) || !plan.persist || plan.pw != 8) return LRBI_ERR_UNSUPPORTED;
     if (!device_status_ptr()) return LRBI_ERR_CUDA;
     const TileRanks none = {nullptr, nullptr, nullptr};
+    if (mn_major) return launch_tc<512, 8, true, true, true, true>(gs, plan, dev, Xt, ip_t, iz_t, dYt, out_rows, dW, dtype, s, nullptr, none, &gi);
     return launch_tc<512, 8, true, true, true>(gs, plan, dev, Xt, ip_t, iz_t, dYt, out_rows, dW, dtype, s, nullptr, none, &gi);
 }
 

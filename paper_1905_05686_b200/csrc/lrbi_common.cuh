@@ -143,7 +143,7 @@ lrbi_status launch_gemm_tc(const Geo &g, const uint16_t *W, const uint32_t *ip, 
                            const TileRanks *ranks = nullptr);   // ranks: one rank per tile (a ranked layout), or null
 
 lrbi_status launch_gemm_tc_dw(const Geo &g, const Geo &gi, const uint16_t *Xt, const uint32_t *ip_t, const uint32_t *iz_t,
-                              const uint16_t *dYt, int out_rows, void *dW, int dtype, cudaStream_t s);
+                              const uint16_t *dYt, int out_rows, void *dW, int dtype, cudaStream_t s, bool mn_major = false);
 
 // Variant that keeps K-split partial sums in the library's fixed device array; allocates nothing.
 lrbi_status launch_gemm_tc_static(const Geo &g, const uint16_t *W, const uint32_t *ip, const uint32_t *iz,

@@ -71,6 +71,12 @@ def test_masked_backward(shape):
             got = b.lrbi_masked_gemm_dw(L, dY, X, ip, iz, dtype=dt, workspace=ws).float().cpu().numpy().astype(np.float64)
             assert rel_fro(got, want_dW) <= tol, ("dW", ws, str(dt), rel_fro(got, want_dW))
             assert not got[M == 0].any()                         # a pruned weight gets no gradient, exactly
+    # aligned layers: one launch, the persistent pair kernel on X and dY as they are (MN-major operands), no copies
+    gr, gc = L.grid
+    if rows % 8 == 0 and cols % 8 == 0 and batch % 8 == 0 and (gc == 1 or tn % 128 == 0) and (gr == 1 or tm % 256 == 0):
+        before = b.launch_count()
+        b.lrbi_masked_gemm_dw(L, dY, X, ip, iz, workspace=None)
+        assert b.launch_count() - before == 1
     assert b.device_status() == 0
 
 
