@@ -42,6 +42,7 @@ NCU_TRAFFIC_BYTES = {
     ("alexnet_fc", -1): 76_200_000,
     ("ffn_16384x4096", -1): 135_800_000,
     ("ffn_16384x4096", -2): 432_300_000,        # dX: 412.4 MB read + 19.9 MB written
+    ("ffn_16384x4096", -3): 409_300_000,        # dW: 295.0 MB read + 114.3 MB written
 }
 # The other configurations, timed after the headline workload and reported in "others" (L2 flushed between calls).
 # batch -1: not the layer's forward pass but the cost evaluation of Algorithm 1's inner loop on its weights and index
