@@ -90,6 +90,86 @@ nmf_prod_z_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict
     }
 }
 
+// The same product for aligned layers (cols % 8 == 0, tn % 8 == 0, k % 4 == 0): the slabs of |W| (32 rows x 128
+// columns) and of Mp (32 rows x 32 rank values) travel through a ring of four shared-memory buffers filled by
+// cp.async three slabs ahead, so nobody waits on device memory inside the loop.
+constexpr int NP_RING = 4;
+constexpr int NP_RING_BYTES = NP_SLAB0 * NP_THREADS * 2 + NP_SLAB0 * NP_KC * 4;      // 8 KB of W + 4 KB of Mp per buffer
+__device__ __forceinline__ void nmf_cp_async_16(void *dst_smem, const void *src, int valid)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src), "r"(valid) : "memory");
+}
+__global__ void __launch_bounds__(NP_THREADS * NP_GROUPS, 2)
+nmf_prod_z_ring_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__ P, float *__restrict__ N1)
+{
+    extern __shared__ __align__(16) uint8_t nmf_ring[];
+    const int tile = blockIdx.y, tr = tile / g.gc, tc = tile - tr * g.gc, k = g.k, t = threadIdx.x, q = threadIdx.y;
+    const int tid = q * NP_THREADS + t;
+    constexpr int RQ = NP_SLAB0 / NP_GROUPS;
+    const int l0 = blockIdx.z * NP_KC, kc = min(NP_KC, k - l0);
+    // a thread owns 4 columns x 8 rank values (lane = group of 4 columns, warp = group of 8 rank values): per row of
+    // the slab it reads 8 bytes of |W| and 32 bytes of Mp for its 32 multiply-adds; with 1 column x 32 rank values it
+    // read 2 + 128 bytes, and the delivery of shared memory to the registers was the limit
+    const int cg = t & 31, lg = t >> 5;
+    const int wrows = min(g.tm, g.rows - tr * g.tm), wcols = min(g.tn, g.cols - tc * g.tn);
+    const uint16_t *Wt = W + (size_t)tr * g.tm * g.cols + (size_t)tc * g.tn;
+    const float *Pt = P + (size_t)tile * g.tm * k;
+    const int nslab = (wrows + NP_SLAB0 - 1) / NP_SLAB0;
+    auto issue = [&](int sl) {                           // (a group is committed even when it is empty: the count stays uniform)
+        if (sl < nslab) {
+            uint8_t *buf = nmf_ring + (sl % NP_RING) * NP_RING_BYTES;
+            const int i0 = sl * NP_SLAB0;
+            {
+                const int r = tid >> 4, c8 = (tid & 15) * 8, jj = blockIdx.x * NP_THREADS + c8;   // 8 columns: all inside the matrix or none
+                const bool in = i0 + r < wrows && jj < wcols;
+                nmf_cp_async_16(reinterpret_cast<uint16_t *>(buf) + r * NP_THREADS + c8, in ? Wt + (size_t)(i0 + r) * g.cols + jj : Wt, in ? 16 : 0);
+            }
+            if (tid < NP_SLAB0 * NP_KC / 4) {
+                const int r = tid >> 3, c4 = (tid & 7) * 4;
+                const bool in = i0 + r < g.tm && c4 < kc;                                         // k % 4 == 0: four values or none
+                nmf_cp_async_16(reinterpret_cast<float *>(buf + NP_SLAB0 * NP_THREADS * 2) + r * NP_KC + c4, in ? Pt + (size_t)(i0 + r) * k + l0 + c4 : Pt, in ? 16 : 0);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    float acc[NP_KC];
+#pragma unroll
+    for (int c = 0; c < NP_KC; ++c) acc[c] = 0.f;
+    for (int sl = 0; sl < NP_RING - 1; ++sl) issue(sl);
+    for (int sl = 0; sl < nslab; ++sl) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(NP_RING - 2) : "memory");   // this thread's part of slab sl has landed
+        __syncthreads();                                 // ... everybody's; and everybody is done with the buffer refilled next
+        issue(sl + NP_RING - 1);
+        const uint8_t *buf = nmf_ring + (sl % NP_RING) * NP_RING_BYTES;
+        const uint16_t *Ws = reinterpret_cast<const uint16_t *>(buf);
+        const float *Ps = reinterpret_cast<const float *>(buf + NP_SLAB0 * NP_THREADS * 2);
+#pragma unroll
+        for (int rr = 0; rr < RQ; ++rr) {
+            const int r = q * RQ + rr;
+            const uint2 wv = *reinterpret_cast<const uint2 *>(Ws + r * NP_THREADS + cg * 4);
+            const float w[4] = {abs_bf16((uint16_t)wv.x), abs_bf16((uint16_t)(wv.x >> 16)), abs_bf16((uint16_t)wv.y), abs_bf16((uint16_t)(wv.y >> 16))};
+            const float4 pa = *reinterpret_cast<const float4 *>(Ps + r * NP_KC + lg * 8);
+            const float4 pb = *reinterpret_cast<const float4 *>(Ps + r * NP_KC + lg * 8 + 4);
+            const float pv[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                for (int ll = 0; ll < 8; ++ll) acc[cc * 8 + ll] = fmaf(pv[ll], w[cc], acc[cc * 8 + ll]);
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    nmf_fold_groups(acc, reinterpret_cast<float *>(nmf_ring), t, q);    // (its first barrier comes before the ring is reused)
+    const int j4 = blockIdx.x * NP_THREADS + cg * 4;    // tn % 8 == 0: the four columns are inside the tile or none is
+    if (q == 0 && j4 < g.tn) {
+        float *Nt = N1 + (size_t)tile * k * g.tn;
+#pragma unroll
+        for (int ll = 0; ll < 8; ++ll) {
+            const int l = l0 + lg * 8 + ll;
+            if (l < k) *reinterpret_cast<float4 *>(Nt + (size_t)l * g.tn + j4) = make_float4(acc[ll], acc[8 + ll], acc[16 + ll], acc[24 + ll]);
+        }
+    }
+}
+
 // N2[i][l] = sum_j |W[i][j]| Z[l][j]   (tm x k per tile; the reduction runs over the tile's columns).
 // grid = (ceil(tm / 128), layer tiles, ceil(k / 32)).  A thread owns row i and 32 values of l.  A slab of 128 rows x 64
 // columns of W goes through shared memory (read along the rows, used along the columns), the slab of Z is stored
@@ -306,8 +386,12 @@ lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, in
     // the update kernels keep k x (threads) old values in shared memory: 128 threads up to rank 64, 32 above
     const unsigned ut = g.k <= 64 ? 128u : 32u;
     const size_t smem_z = (size_t)g.k * ut * sizeof(float), smem_p = (size_t)ut * (g.k + 1) * sizeof(float);
+    // aligned layers: the product kernels that stream their slabs through a cp.async ring
+    const bool ring = (g.cols % 8) == 0 && (g.tn % 8) == 0 && (g.k % 4) == 0 &&
+                      ((reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(mp) | reinterpret_cast<uintptr_t>(mz)) & 15u) == 0;
     for (int it = 0; it < iterations; ++it) {
-        nmf_prod_z_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mp, N);
+        if (ring) nmf_prod_z_ring_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), NP_RING * NP_RING_BYTES, s>>>(g, W, mp, N);
+        else nmf_prod_z_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mp, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
         nmf_gram_kernel<0><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tm + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mp, G);
         nmf_update_z_kernel<<<dim3((unsigned)((g.tn + ut - 1) / ut), (unsigned)tiles), ut, smem_z, s>>>(g, N, G, mz, eps);
