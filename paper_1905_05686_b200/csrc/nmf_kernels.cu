@@ -8,6 +8,8 @@
 //                 (a thread owns one output column / row and 32 rank values; |W| is read once per 32 rank values)
 //   nmf_gram      G  = Mp^T Mp  or  Mz Mz^T   (k x k per tile)
 //   nmf_update_z / nmf_update_p   the element-wise update with the k-term denominator
+#include <mutex>
+
 #include "lrbi_common.cuh"
 
 namespace lrbi {
@@ -242,6 +244,93 @@ nmf_prod_p_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict
     }
 }
 
+// The ring version of the second product (same conditions as nmf_prod_z_ring_kernel): slabs of 128 rows x 64 columns of
+// |W| (rows 144 bytes apart) and of 64 columns x 32 rank values of Mz (stored [column][rank value], filled by 4-byte
+// cp.async), three buffers.  A thread owns rows rg, rg + 32, rg + 64, rg + 96 and 8 rank values.
+constexpr int NP_RING1 = 3;
+constexpr int NP_WPITCH = NP_SLAB1 + 8;                  // bf16 per staged row of W: 144 bytes
+constexpr int NP_RING1_BYTES = NP_THREADS * NP_WPITCH * 2 + NP_SLAB1 * NP_KC * 4;
+__global__ void __launch_bounds__(NP_THREADS * NP_GROUPS, 2)
+nmf_prod_p_ring_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__ Z, float *__restrict__ N2)
+{
+    extern __shared__ __align__(16) uint8_t nmf_ring[];
+    const int tile = blockIdx.y, tr = tile / g.gc, tc = tile - tr * g.gc, k = g.k, t = threadIdx.x, q = threadIdx.y;
+    const int tid = q * NP_THREADS + t;
+    const int ib = blockIdx.x * NP_THREADS, l0 = blockIdx.z * NP_KC, kc = min(NP_KC, k - l0);
+    const int rg = t & 31, lg = t >> 5;
+    const int wrows = min(g.tm, g.rows - tr * g.tm), wcols = min(g.tn, g.cols - tc * g.tn);
+    const uint16_t *Wt = W + (size_t)tr * g.tm * g.cols + (size_t)tc * g.tn;
+    const float *Zt = Z + (size_t)tile * k * g.tn;
+    const int nslab = (wcols + NP_SLAB1 - 1) / NP_SLAB1;
+    auto issue = [&](int sl) {
+        if (sl < nslab) {
+            uint8_t *buf = nmf_ring + (sl % NP_RING1) * NP_RING1_BYTES;
+            const int j0 = sl * NP_SLAB1;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {                // 128 rows x 8 pieces of 8 columns
+                const int e = tid + NP_THREADS * NP_GROUPS * u, r = e >> 3, c8 = (e & 7) * 8;
+                const bool in = ib + r < wrows && j0 + c8 < wcols;
+                nmf_cp_async_16(reinterpret_cast<uint16_t *>(buf) + r * NP_WPITCH + c8, in ? Wt + (size_t)(ib + r) * g.cols + j0 + c8 : Wt, in ? 16 : 0);
+            }
+            float *Zs = reinterpret_cast<float *>(buf + NP_THREADS * NP_WPITCH * 2);
+#pragma unroll
+            for (int u = 0; u < NP_KC * NP_SLAB1 / (NP_THREADS * NP_GROUPS); ++u) {
+                const int e = tid + NP_THREADS * NP_GROUPS * u, c = e / NP_SLAB1, jj = e - c * NP_SLAB1;
+                const bool in = c < kc && j0 + jj < g.tn;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(Zs + jj * NP_KC + c)),
+                             "l"(in ? Zt + (size_t)(l0 + c) * g.tn + j0 + jj : Zt), "r"(in ? 4 : 0) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    float acc[NP_KC];
+#pragma unroll
+    for (int c = 0; c < NP_KC; ++c) acc[c] = 0.f;
+    for (int sl = 0; sl < NP_RING1 - 1; ++sl) issue(sl);
+    constexpr int JQ = NP_SLAB1 / NP_GROUPS;            // columns of a slab per thread: 16, two pieces of 8
+    for (int sl = 0; sl < nslab; ++sl) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(NP_RING1 - 2) : "memory");
+        __syncthreads();
+        issue(sl + NP_RING1 - 1);
+        const uint8_t *buf = nmf_ring + (sl % NP_RING1) * NP_RING1_BYTES;
+        const uint16_t *Ws = reinterpret_cast<const uint16_t *>(buf);
+        const float *Zs = reinterpret_cast<const float *>(buf + NP_THREADS * NP_WPITCH * 2);
+#pragma unroll
+        for (int pc = 0; pc < JQ / 8; ++pc) {
+            const int jb = q * JQ + pc * 8;
+            uint4 wv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) wv[u] = *reinterpret_cast<const uint4 *>(Ws + (rg + 32 * u) * NP_WPITCH + jb);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float4 za = *reinterpret_cast<const float4 *>(Zs + (jb + e) * NP_KC + lg * 8);
+                const float4 zb = *reinterpret_cast<const float4 *>(Zs + (jb + e) * NP_KC + lg * 8 + 4);
+                const float zv[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t word = e < 2 ? wv[u].x : e < 4 ? wv[u].y : e < 6 ? wv[u].z : wv[u].w;
+                    const float w = abs_bf16((uint16_t)((e & 1) ? word >> 16 : word));
+#pragma unroll
+                    for (int ll = 0; ll < 8; ++ll) acc[u * 8 + ll] = fmaf(w, zv[ll], acc[u * 8 + ll]);
+                }
+            }
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    nmf_fold_groups(acc, reinterpret_cast<float *>(nmf_ring), t, q);
+    if (q == 0) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = ib + rg + 32 * u;
+            if (i < g.tm) {
+                float *Nt = N2 + ((size_t)tile * g.tm + i) * k + l0 + lg * 8;      // k % 4 == 0: 16-byte aligned
+                if (lg * 8 < kc) *reinterpret_cast<float4 *>(Nt) = make_float4(acc[u * 8], acc[u * 8 + 1], acc[u * 8 + 2], acc[u * 8 + 3]);
+                if (lg * 8 + 4 < kc) *reinterpret_cast<float4 *>(Nt + 4) = make_float4(acc[u * 8 + 4], acc[u * 8 + 5], acc[u * 8 + 6], acc[u * 8 + 7]);
+            }
+        }
+    }
+}
+
 // G[a][b] = sum_r F(r, a) F(r, b): ZMODE 0: F = Mp [tm][k] (r = row), ZMODE 1: F = Mz [k][tn] (r = column).
 // grid = (blocks of 32 x 32 entries, layer tiles, slices of 64 values of r): a block stages its slice of the two
 // 32-wide strips of F in shared memory, a thread sums four entries and adds them to G (zeroed before the launch)
@@ -389,13 +478,25 @@ lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, in
     // aligned layers: the product kernels that stream their slabs through a cp.async ring
     const bool ring = (g.cols % 8) == 0 && (g.tn % 8) == 0 && (g.k % 4) == 0 &&
                       ((reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(mp) | reinterpret_cast<uintptr_t>(mz)) & 15u) == 0;
+    if (ring) {
+        int dev = 0;
+        static bool attr_done[LRBI_MAX_DEVICES] = {false};
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= LRBI_MAX_DEVICES) return LRBI_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(lib_mutex());
+        if (!attr_done[dev]) {                           // more than 48 KB of dynamic shared memory: a per-device opt-in
+            const cudaError_t ea = cudaFuncSetAttribute(nmf_prod_p_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NP_RING1 * NP_RING1_BYTES);
+            if (ea != cudaSuccess) { note_cuda_error((int)ea); return LRBI_ERR_CUDA; }
+            attr_done[dev] = true;
+        }
+    }
     for (int it = 0; it < iterations; ++it) {
         if (ring) nmf_prod_z_ring_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), NP_RING * NP_RING_BYTES, s>>>(g, W, mp, N);
         else nmf_prod_z_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mp, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
         nmf_gram_kernel<0><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tm + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mp, G);
         nmf_update_z_kernel<<<dim3((unsigned)((g.tn + ut - 1) / ut), (unsigned)tiles), ut, smem_z, s>>>(g, N, G, mz, eps);
-        nmf_prod_p_kernel<<<dim3((unsigned)((g.tm + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mz, N);
+        if (ring) nmf_prod_p_ring_kernel<<<dim3((unsigned)((g.tm + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), NP_RING1 * NP_RING1_BYTES, s>>>(g, W, mz, N);
+        else nmf_prod_p_kernel<<<dim3((unsigned)((g.tm + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mz, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
         nmf_gram_kernel<1><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tn + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mz, G);
         nmf_update_p_kernel<<<dim3((unsigned)((g.tm + ut - 1) / ut), (unsigned)tiles), ut, smem_p, s>>>(g, N, G, mp, eps);
