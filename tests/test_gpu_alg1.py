@@ -146,3 +146,22 @@ def test_search_driven_by_the_gpu_kernels_matches_the_oracle_search():
         assert got[0] == pytest.approx(want["Sp"]) and got[1] == want["Sz"] and got[4] == want["lost"]
         assert got[2] == pytest.approx(want["cost"], rel=1e-6) and got[3] == want["Sa"]
     assert best[0] == pytest.approx(ref["best"]["Sp"]) and best[1] == ref["best"]["Sz"]
+
+
+@pytest.mark.parametrize("name", ["alexnet_fc", "ffn_16384x4096"])
+def test_index_cost_at_the_benchmark_sizes(name):
+    """The two layers `bench.py` times the cost evaluation on, whole: every tile's counts exactly, its cost to 1e-6."""
+    b = _b()
+    L = synth.CONFIGS[name]
+    Ip, Iz = synth.make_factors(L)
+    Wb = synth.make_weights(L)
+    theta = float(np.float32(1.3 * L.w_std))
+    Ia = oracle.decode_mask(Ip, Iz, L.rows, L.cols)
+    kept_i, kept_a, lost, cost = oracle.index_cost(Wb, theta, Ia, L.tile_rows, L.tile_cols)
+    out = b.lrbi_index_cost(L, b.to_device_bf16(Wb), theta, b.to_device_words(synth.pack_ip(Ip)), b.to_device_words(synth.pack_iz(Iz)))
+    torch.cuda.synchronize()
+    g_i, g_a, g_l, g_c = b.tile_costs(out)
+    assert kept_i.sum() > 0 and lost.sum() > 0                   # the threshold cuts inside the distribution
+    assert (g_i == kept_i).all() and (g_a == kept_a).all() and (g_l == lost).all()
+    assert np.allclose(g_c, cost, rtol=1e-6, atol=0)
+    assert b.device_status() == 0

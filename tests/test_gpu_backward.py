@@ -94,3 +94,38 @@ def test_poisoned_pruned_weights_do_not_reach_dx():
     Wt = b.lrbi_transpose_bf16(b.to_device_bf16(Wb2))
     got = b.lrbi_masked_gemm_dx(L, Wt, ip, iz, b.to_device_bf16(dYb)).float().cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all() and rel_fro(got, want) <= TOL
+
+
+def test_backward_at_the_benchmark_size_on_sampled_rows():
+    """dX and dW of the FFN layer at batch 4096, the calls `bench.py` times (dX on the persistent pair kernel, dW on
+    the same kernel with MN-major operands, one launch).  A row of dX depends on one row of dY and a row of dW on one
+    column of dY, so the oracle computes a sample of rows of each from the matching slices of the inputs."""
+    b = _b()
+    L = synth.CONFIGS["ffn_16384x4096"]
+    batch = 4096
+    Ip, Iz = synth.make_factors(L)
+    M = oracle.decode_mask(Ip, Iz, L.rows, L.cols)
+    Wb, Xb = synth.make_weights(L), synth.make_activations(L, batch)
+    dYb = synth.make_activations(synth.Layer("bwd_dy", L.cols, L.rows, L.tile_cols, L.tile_rows, L.rank, 0.2, 0.02), batch)   # [batch, rows]
+    ip, iz = b.to_device_words(synth.pack_ip(Ip)), b.to_device_words(synth.pack_iz(Iz))
+    W, X, dY = b.to_device_bf16(Wb), b.to_device_bf16(Xb), b.to_device_bf16(dYb)
+    rng = np.random.default_rng(7)
+    # --- dX: sampled batch rows (first and last included)
+    bs = np.unique(np.concatenate([[0, batch - 1], rng.integers(0, batch, 22)]))
+    want_dX, _ = oracle.masked_backward(Wb, M, Xb[bs], dYb[bs])
+    Wt = b.lrbi_transpose_bf16(W)
+    before = b.launch_count()
+    got = b.lrbi_masked_gemm_dx(L, Wt, ip, iz, dY, dtype=torch.float32)
+    assert b.launch_count() - before == 1
+    assert rel_fro(got[torch.from_numpy(bs).cuda()].cpu().numpy().astype(np.float64), want_dX) <= TOL_F32
+    del got, Wt
+    # --- dW: sampled rows of the layer, from every tile row and both CTAs of a pair
+    os_ = np.unique(np.concatenate([[0, 127, 128, 255, 256, L.rows - 1], rng.integers(0, L.rows, 26)]))
+    _, want_dW = oracle.masked_backward(Wb[os_], M[os_], Xb, np.ascontiguousarray(dYb[:, os_]))
+    before = b.launch_count()
+    got = b.lrbi_masked_gemm_dw(L, dY, X, ip, iz, dtype=torch.float32, workspace=None)
+    assert b.launch_count() - before == 1
+    got = got[torch.from_numpy(os_).cuda()].cpu().numpy().astype(np.float64)
+    assert rel_fro(got, want_dW) <= TOL_F32
+    assert not got[M[os_] == 0].any()
+    assert b.device_status() == 0

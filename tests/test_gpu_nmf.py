@@ -60,3 +60,23 @@ def test_one_step_by_hand_and_pipeline_into_the_packed_factors():
     ip, iz = b.lrbi_threshold_pack(L, mp, mz, one(1.0), one(2.0))     # Ip = (0, 1)^T, Iz = (0, 1): only |W| = 4 is kept
     mask = b.lrbi_decode_mask(L, ip, iz).cpu().numpy().view(np.uint32)
     assert mask.ravel().tolist() == [0, 2]
+
+
+def test_nmf_at_the_benchmark_size():
+    """Two iterations on the AlexNet layer (144 tiles of 512 x 512, k = 32), the configuration `bench.py` times; this
+    is the shape that runs on the cp.async ring kernels."""
+    b = _b()
+    L = synth.CONFIGS["alexnet_fc"]
+    tiles = L.grid[0] * L.grid[1]
+    rng = np.random.default_rng(11)
+    Wb = synth.make_weights(L)
+    Mp0 = (rng.random((tiles, L.tile_rows, L.rank)) * 0.1 + 0.01).astype(np.float32)
+    Mz0 = (rng.random((tiles, L.rank, L.tile_cols)) * 0.1 + 0.01).astype(np.float32)
+    want_p, want_z = oracle.nmf_multiplicative(Wb, Mp0, Mz0, L.tile_rows, L.tile_cols, 2)
+    mp, mz = torch.from_numpy(Mp0.copy()).cuda(), torch.from_numpy(Mz0.copy()).cuda()
+    b.lrbi_nmf_update(L, b.to_device_bf16(Wb), mp, mz, 2)
+    torch.cuda.synchronize()
+    for got, want in ((mp.cpu().numpy().astype(np.float64), want_p), (mz.cpu().numpy().astype(np.float64), want_z)):
+        assert np.isfinite(got).all() and (got >= 0).all()
+        assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 2e-4
+    assert b.device_status() == 0
