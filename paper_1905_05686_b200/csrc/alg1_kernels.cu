@@ -104,7 +104,9 @@ __device__ __forceinline__ void cost_element(uint32_t wbits, bool ia, float thet
 
 // FAST: cols % 8 == 0, tn % 32 == 0 (or one tile column with cols % 32 == 0 handled by zero planes), planes fit shared memory.
 // grid = (bands per tile, tiles).  Shared memory: planes[kw*32][tnw] (FAST only).
-template <bool FAST>
+// U: 256-column chunks of a row that a warp takes at a time (a tile of 512 columns has two: four would leave half
+// of every step idle).
+template <bool FAST, int U>
 __global__ void __launch_bounds__(A1_THREADS)
 index_cost_kernel(Geo g, const uint16_t *__restrict__ W, float theta, const uint32_t *__restrict__ ip,
                   const uint32_t *__restrict__ iz, lrbi_tile_cost *__restrict__ out)
@@ -142,23 +144,25 @@ index_cost_kernel(Geo g, const uint16_t *__restrict__ W, float theta, const uint
                        : make_uint4(0, 0, 0, 0);
         };
         uint32_t n_i = 0, n_a = 0, n_l = 0;
-        // groups of four chunks (1024 columns of a row): a warp keeps 2 KB requested ahead of what it evaluates
-        const int ngr = (nch + 3) >> 2;
-        uint4 wnext[4];
+        // groups of U chunks (U * 256 columns of a row): a warp keeps U * 512 bytes requested ahead of what it evaluates
+        const int ngr = (nch + U - 1) / U;
+        uint4 wnext[U];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) wnext[u] = load_w(0, u);
+        for (int u = 0; u < U; ++u) wnext[u] = load_w(0, u);
         for (int j = 0; j < nrows_w; ++j) {
             const int i = i_begin + warp + j * (A1_THREADS / 32);
             const uint32_t *ipw = ip + ((size_t)tile * g.tm + i) * g.kw;
             for (int gr4 = 0; gr4 < ngr; ++gr4) {
-                uint4 v[4];
+                uint4 v[U];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) v[u] = wnext[u];
+                for (int u = 0; u < U; ++u) v[u] = wnext[u];
                 const int jn = gr4 + 1 < ngr ? j : j + 1, gn = gr4 + 1 < ngr ? gr4 + 1 : 0;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) wnext[u] = load_w(jn, gn * 4 + u);
-                uint32_t bits[4] = {0u, 0u, 0u, 0u};                        // index bits of the words that hold this lane's columns
-                const int word0 = gr4 * 32 + (lane >> 2);                   // chunk u: word0 + 8 u
+                for (int u = 0; u < U; ++u) wnext[u] = load_w(jn, gn * U + u);
+                uint32_t bits[U];                                           // index bits of the words that hold this lane's columns
+#pragma unroll
+                for (int u = 0; u < U; ++u) bits[u] = 0u;
+                const int word0 = gr4 * (8 * U) + (lane >> 2);              // chunk u: word0 + 8 u
                 for (int lb = 0; lb < g.kw; ++lb) {
                     uint32_t x = __ldg(ipw + lb);                           // warp-uniform: no divergence below
                     if (lb == g.kw - 1) x &= tail;
@@ -166,18 +170,16 @@ index_cost_kernel(Geo g, const uint16_t *__restrict__ W, float theta, const uint
                         const uint32_t *pl = a1_planes + (lb * 32 + __ffs(x) - 1) * tnw;
                         x &= x - 1;
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) bits[u] |= pl[min(word0 + 8 * u, tnw - 1)];
+                        for (int u = 0; u < U; ++u) bits[u] |= pl[min(word0 + 8 * u, tnw - 1)];
                     }
                 }
+                float cf = 0.f;                                             // fp32 over the group's 8 U weights, fp64 beyond
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = (gr4 * 4 + u) * 256 + lane * 8;
-                    if (c < ncols) {
-                        float cf = 0.f;
-                        cost_chunk(v[u], bits[u] >> (c & 31), theta, n_i, n_a, n_l, cf);
-                        acc.cost += (double)cf;
-                    }
+                for (int u = 0; u < U; ++u) {
+                    const int c = (gr4 * U + u) * 256 + lane * 8;
+                    if (c < ncols) cost_chunk(v[u], bits[u] >> (c & 31), theta, n_i, n_a, n_l, cf);
                 }
+                acc.cost += (double)cf;
             }
         }
         acc.kept_i = n_i; acc.kept_a = n_a; acc.lost = n_l;
@@ -235,8 +237,11 @@ lrbi_status launch_index_cost(const Geo &g, const uint16_t *W, float theta, cons
     const size_t smem = (size_t)g.kw * 32 * tnw * sizeof(uint32_t);
     const bool fast = (g.cols % 8) == 0 && (g.tn % 8) == 0 && smem <= 48 * 1024;
     dim3 grid((unsigned)((g.tm + A1_BAND - 1) / A1_BAND), (unsigned)tiles);
-    if (fast) index_cost_kernel<true><<<grid, A1_THREADS, smem, s>>>(g, W, theta, ip, iz, out);
-    else index_cost_kernel<false><<<grid, A1_THREADS, 0, s>>>(g, W, theta, ip, iz, out);
+    const int nch = (g.tn + 255) / 256;                  // 256-column chunks of a tile row
+    if (fast && nch <= 1) index_cost_kernel<true, 1><<<grid, A1_THREADS, smem, s>>>(g, W, theta, ip, iz, out);
+    else if (fast && nch == 2) index_cost_kernel<true, 2><<<grid, A1_THREADS, smem, s>>>(g, W, theta, ip, iz, out);
+    else if (fast) index_cost_kernel<true, 4><<<grid, A1_THREADS, smem, s>>>(g, W, theta, ip, iz, out);
+    else index_cost_kernel<false, 1><<<grid, A1_THREADS, 0, s>>>(g, W, theta, ip, iz, out);
     count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess) { note_cuda_error((int)e); return LRBI_ERR_CUDA; }

@@ -1,6 +1,6 @@
 """Inner loop of Algorithm 1 on the GPU (binary conversion into packed factors, per-tile index counts and
 cost) against the CPU oracle, through the C ABI.  Bits and counts must agree exactly; the cost is a sum of
-bf16 magnitudes accumulated in fp32 over 8 weights and in fp64 beyond, held to 1e-6 relative."""
+bf16 magnitudes accumulated in fp32 over up to 32 weights and in fp64 beyond, held to 1e-6 relative."""
 import os
 
 import numpy as np
