@@ -376,12 +376,17 @@ constexpr int NMF_MAX_RANK = 256;
 // memory ([k][columns]); a thread owns column j and forms four denominators at a time, reading row m of the
 // (symmetric) Gram matrix as G1[m][l .. l+3].
 __global__ void
-nmf_update_z_kernel(Geo g, const float *__restrict__ N1, const float *__restrict__ G1, float *__restrict__ Z, float eps)
+nmf_update_z_kernel(Geo g, const float *__restrict__ N1, const float *__restrict__ G1, float *__restrict__ Z, float eps, int gram_in_smem)
 {
-    extern __shared__ __align__(16) float nmf_old[];    // [k][blockDim.x]
+    extern __shared__ __align__(16) float nmf_old[];    // [k][blockDim.x], then (gram_in_smem) the tile's Gram matrix [k][k]
     const int tile = blockIdx.y, k = g.k, t = threadIdx.x, nb = blockDim.x, j = blockIdx.x * nb + t;
     float *Zt = Z + (size_t)tile * k * g.tn;
     const float *Nt = N1 + (size_t)tile * k * g.tn, *Gt = G1 + (size_t)tile * k * k;
+    if (gram_in_smem) {                                  // the sums below then wait on shared memory, not on L1 / L2
+        float *Gs = nmf_old + k * nb;
+        for (int e = t; e < k * k; e += nb) Gs[e] = Gt[e];
+        Gt = Gs;
+    }
     for (int m0 = 0; m0 < k; m0 += 8) {                  // eight requests in flight per thread
         float v[8];
 #pragma unroll
@@ -402,13 +407,13 @@ nmf_update_z_kernel(Geo g, const float *__restrict__ N1, const float *__restrict
         for (int m = 0; m < k; ++m) {
             const float z = nmf_old[m * nb + t];
             if (vec) {
-                const float4 gv = __ldg(reinterpret_cast<const float4 *>(Gt + (size_t)m * k + l0));
+                const float4 gv = *reinterpret_cast<const float4 *>(Gt + (size_t)m * k + l0);
                 den[0] = fmaf(gv.x, z, den[0]); den[1] = fmaf(gv.y, z, den[1]);
                 den[2] = fmaf(gv.z, z, den[2]); den[3] = fmaf(gv.w, z, den[3]);
             } else {
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (l0 + u < k) den[u] = fmaf(__ldg(Gt + (size_t)(l0 + u) * k + m), z, den[u]);
+                    if (l0 + u < k) den[u] = fmaf(Gt[(size_t)(l0 + u) * k + m], z, den[u]);
             }
         }
 #pragma unroll
@@ -420,12 +425,17 @@ nmf_update_z_kernel(Geo g, const float *__restrict__ N1, const float *__restrict
 // Mp[i][l] *= N2[i][l] / (sum_m Mp[i][m] G2[m][l] + eps).  The block's rows of Mp (contiguous in memory) are staged in
 // shared memory, k + 1 words apart; a thread owns row i.
 __global__ void
-nmf_update_p_kernel(Geo g, const float *__restrict__ N2, const float *__restrict__ G2, float *__restrict__ P, float eps)
+nmf_update_p_kernel(Geo g, const float *__restrict__ N2, const float *__restrict__ G2, float *__restrict__ P, float eps, int gram_in_smem)
 {
-    extern __shared__ __align__(16) float nmf_old[];    // [blockDim.x][k + 1]
+    extern __shared__ __align__(16) float nmf_old[];    // [blockDim.x][k + 1], then (gram_in_smem) the Gram matrix [k][k], 16-byte aligned
     const int tile = blockIdx.y, k = g.k, t = threadIdx.x, nb = blockDim.x, ib = blockIdx.x * nb, i = ib + t;
     float *Pt = P + (size_t)tile * g.tm * k;
     const float *Nt = N2 + (size_t)tile * g.tm * k, *Gt = G2 + (size_t)tile * k * k;
+    if (gram_in_smem) {
+        float *Gs = nmf_old + ((nb * (k + 1) + 3) & ~3);
+        for (int e = t; e < k * k; e += nb) Gs[e] = Gt[e];
+        Gt = Gs;
+    }
     const int nrows = min(nb, g.tm - ib);
     for (int e = t; e < nrows * k; e += nb) {
         const int r = e / k, c = e - r * k;
@@ -444,13 +454,13 @@ nmf_update_p_kernel(Geo g, const float *__restrict__ N2, const float *__restrict
         for (int m = 0; m < k; ++m) {
             const float p = mine[m];
             if (vec) {
-                const float4 gv = __ldg(reinterpret_cast<const float4 *>(Gt + (size_t)m * k + l0));
+                const float4 gv = *reinterpret_cast<const float4 *>(Gt + (size_t)m * k + l0);
                 den[0] = fmaf(p, gv.x, den[0]); den[1] = fmaf(p, gv.y, den[1]);
                 den[2] = fmaf(p, gv.z, den[2]); den[3] = fmaf(p, gv.w, den[3]);
             } else {
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (l0 + u < k) den[u] = fmaf(p, __ldg(Gt + (size_t)m * k + l0 + u), den[u]);
+                    if (l0 + u < k) den[u] = fmaf(p, Gt[(size_t)m * k + l0 + u], den[u]);
             }
         }
 #pragma unroll
@@ -474,7 +484,10 @@ lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, in
     const unsigned kc = (unsigned)((g.k + NP_KC - 1) / NP_KC), kb = (unsigned)((g.k + 31) / 32);
     // the update kernels keep k x (threads) old values in shared memory: 128 threads up to rank 64, 32 above
     const unsigned ut = g.k <= 64 ? 128u : 32u;
-    const size_t smem_z = (size_t)g.k * ut * sizeof(float), smem_p = (size_t)ut * (g.k + 1) * sizeof(float);
+    // the Gram matrix of a tile beside the old values in shared memory, where both fit the 48 KB a launch gets without opt-in
+    const int gsm = ((((size_t)ut * (g.k + 1) + 3) & ~(size_t)3) + (size_t)g.k * g.k) * sizeof(float) <= 48 * 1024 ? 1 : 0;
+    const size_t gbytes = gsm ? (size_t)g.k * g.k * sizeof(float) : 0;
+    const size_t smem_z = (size_t)g.k * ut * sizeof(float) + gbytes, smem_p = (((size_t)ut * (g.k + 1) + 3) & ~(size_t)3) * sizeof(float) + gbytes;
     // aligned layers: the product kernels that stream their slabs through a cp.async ring
     const bool ring = (g.cols % 8) == 0 && (g.tn % 8) == 0 && (g.k % 4) == 0 &&
                       ((reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(mp) | reinterpret_cast<uintptr_t>(mz)) & 15u) == 0;
@@ -494,12 +507,12 @@ lrbi_status launch_nmf(const Geo &g, const uint16_t *W, float *mp, float *mz, in
         else nmf_prod_z_kernel<<<dim3((unsigned)((g.tn + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mp, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
         nmf_gram_kernel<0><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tm + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mp, G);
-        nmf_update_z_kernel<<<dim3((unsigned)((g.tn + ut - 1) / ut), (unsigned)tiles), ut, smem_z, s>>>(g, N, G, mz, eps);
+        nmf_update_z_kernel<<<dim3((unsigned)((g.tn + ut - 1) / ut), (unsigned)tiles), ut, smem_z, s>>>(g, N, G, mz, eps, gsm);
         if (ring) nmf_prod_p_ring_kernel<<<dim3((unsigned)((g.tm + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), NP_RING1 * NP_RING1_BYTES, s>>>(g, W, mz, N);
         else nmf_prod_p_kernel<<<dim3((unsigned)((g.tm + NP_THREADS - 1) / NP_THREADS), (unsigned)tiles, kc), dim3(NP_THREADS, NP_GROUPS), 0, s>>>(g, W, mz, N);
         cudaMemsetAsync(G, 0, (size_t)tiles * g.k * g.k * sizeof(float), s);
         nmf_gram_kernel<1><<<dim3(kb * kb, (unsigned)tiles, (unsigned)((g.tn + NMF_GRAM_SLICE - 1) / NMF_GRAM_SLICE)), 256, 0, s>>>(g, mz, G);
-        nmf_update_p_kernel<<<dim3((unsigned)((g.tm + ut - 1) / ut), (unsigned)tiles), ut, smem_p, s>>>(g, N, G, mp, eps);
+        nmf_update_p_kernel<<<dim3((unsigned)((g.tm + ut - 1) / ut), (unsigned)tiles), ut, smem_p, s>>>(g, N, G, mp, eps, gsm);
         count_launch(6);
     }
     const cudaError_t e = cudaGetLastError();
