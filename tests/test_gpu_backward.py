@@ -40,6 +40,8 @@ SHAPES = [
     (1024, 768, 512, 128, 64, 520),
     (384, 776, 384, 776, 256, 40),        # one tile
     (512, 2048, 256, 1024, 145, 136),
+    (1000, 1304, 1000, 1304, 20, 72),     # one tile, nothing a multiple of 64: ragged 64 x 64 boxes of the MN-major dW on every side
+    (2048, 520, 512, 520, 9, 1032),       # dW tiles of 256 x 512 outputs with a ragged third row pair; K = 16 blocks + 8
 ]
 
 
