@@ -249,7 +249,8 @@ nmf_prod_p_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict
 // cp.async), three buffers.  A thread owns rows rg, rg + 32, rg + 64, rg + 96 and 8 rank values.
 constexpr int NP_RING1 = 3;
 constexpr int NP_WPITCH = NP_SLAB1 + 8;                  // bf16 per staged row of W: 144 bytes
-constexpr int NP_RING1_BYTES = NP_THREADS * NP_WPITCH * 2 + NP_SLAB1 * NP_KC * 4;
+constexpr int NP_ZPITCH = NP_KC + 4;                     // floats per staged column of Mz: the 4-byte copies of 32 columns spread over 8 banks, not 1
+constexpr int NP_RING1_BYTES = NP_THREADS * NP_WPITCH * 2 + NP_SLAB1 * NP_ZPITCH * 4;
 __global__ void __launch_bounds__(NP_THREADS * NP_GROUPS, 2)
 nmf_prod_p_ring_kernel(Geo g, const uint16_t *__restrict__ W, const float *__restrict__ Z, float *__restrict__ N2)
 {
@@ -277,7 +278,7 @@ nmf_prod_p_ring_kernel(Geo g, const uint16_t *__restrict__ W, const float *__res
             for (int u = 0; u < NP_KC * NP_SLAB1 / (NP_THREADS * NP_GROUPS); ++u) {
                 const int e = tid + NP_THREADS * NP_GROUPS * u, c = e / NP_SLAB1, jj = e - c * NP_SLAB1;
                 const bool in = c < kc && j0 + jj < g.tn;
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(Zs + jj * NP_KC + c)),
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(Zs + jj * NP_ZPITCH + c)),
                              "l"(in ? Zt + (size_t)(l0 + c) * g.tn + j0 + jj : Zt), "r"(in ? 4 : 0) : "memory");
             }
         }
@@ -303,8 +304,8 @@ nmf_prod_p_ring_kernel(Geo g, const uint16_t *__restrict__ W, const float *__res
             for (int u = 0; u < 4; ++u) wv[u] = *reinterpret_cast<const uint4 *>(Ws + (rg + 32 * u) * NP_WPITCH + jb);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const float4 za = *reinterpret_cast<const float4 *>(Zs + (jb + e) * NP_KC + lg * 8);
-                const float4 zb = *reinterpret_cast<const float4 *>(Zs + (jb + e) * NP_KC + lg * 8 + 4);
+                const float4 za = *reinterpret_cast<const float4 *>(Zs + (jb + e) * NP_ZPITCH + lg * 8);
+                const float4 zb = *reinterpret_cast<const float4 *>(Zs + (jb + e) * NP_ZPITCH + lg * 8 + 4);
                 const float zv[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
